@@ -1,0 +1,247 @@
+"""fp64 CPU oracle for the OAPL LM-head hot path.  TEST INFRASTRUCTURE ONLY.
+
+This module is the plain, slow, obviously-correct statement of what the CUDA
+library computes.  It is imported only by the tests, by the smoke check and by
+the benchmark's CPU-baseline leg; the product path never calls it and shares no
+code with it.  Everything is float64 numpy; the only library primitive used as
+a step is the dense matrix product.
+
+What it states (OAPL paper, "Method" section):
+
+* token log-probability  ln pi(y_t | x, y_<t) = z[y_t] - ln sum_v exp z[v] with
+  z = h . W^T  (the policy's next-token distribution; the sequence quantity
+  pi(y|x) of Eq. 3 is the product over the response tokens, so its log is the
+  masked sum of the token log-probabilities);
+* the group value estimate of Eq. 2, V^(x) = beta ln (1/G) sum_i exp(r_i/beta);
+* the optimal-advantage estimate A_i = r_i - V^(x) (text below Eq. 2);
+* the squared-regression objective of Eq. 3 with the two temperatures of the
+  "Experimental Setup" section (beta_v in Eq. 2, beta_loss in Eq. 3);
+* its gradient with respect to the hidden states H and the LM-head weight W,
+  obtained by differentiating Eq. 3 through the softmax (Algorithm 1 performs
+  gradient descent on Eq. 3; no gradient flows through V^ or through the
+  inference engine's log-probabilities, which are data).
+
+Pins (tests/test_oracle_pins.py): brute-force logits by explicit loops, softmax
+normalisation, the W=0 and V=2 closed forms, scipy's logsumexp, the beta->0 and
+beta->inf limits of Eq. 2, its binary-reward closed form and a 60-digit decimal
+evaluation of the literal formula, zero loss and zero gradient at the
+closed-form optimum, central finite differences of the loss, and the zero
+column sum of dW.  The paper prints no worked numeric example, so the numeric
+end-to-end value of a whole step is "parity unpinned" beyond those pins.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# input decoding
+# --------------------------------------------------------------------------
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bfloat16 bit patterns (uint16) to float64 exactly.
+
+    A bfloat16 is the upper half of an IEEE float32, so placing the 16 bits in
+    the high half of a 32-bit word and reading it as float32 is exact, and
+    float32 -> float64 is exact.
+    """
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    as_f32 = (bits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    return as_f32.astype(np.float64)
+
+
+# --------------------------------------------------------------------------
+# token and sequence log-probabilities
+# --------------------------------------------------------------------------
+def logits(H: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """z[n, v] = sum_k H[n, k] * W[v, k]   (LM head without bias)."""
+    return np.asarray(H, dtype=np.float64) @ np.asarray(W, dtype=np.float64).T
+
+
+def log_sum_exp(z: np.ndarray) -> np.ndarray:
+    """Row-wise natural-log ln sum_v exp z[n, v], shifted by the row maximum."""
+    M = z.max(axis=1)
+    return M + np.log(np.exp(z - M[:, None]).sum(axis=1))
+
+
+def token_logprobs(H, W, targets, mask):
+    """Per-row ln pi(target | prefix) and the row's log-sum-exp.
+
+    H [N, d], W [V, d] float64; targets [N] int; mask [N] in {0,1}.
+    Rows with mask == 0 give lp = 0 and lse = 0 and their target is ignored.
+    Returns (lp [N], lse [N]).
+    """
+    H = np.asarray(H, dtype=np.float64)
+    N = H.shape[0]
+    mask = np.asarray(mask).astype(bool)
+    targets = np.asarray(targets).astype(np.int64)
+    lp = np.zeros(N)
+    lse = np.zeros(N)
+    live = np.flatnonzero(mask)
+    if live.size:
+        z = logits(H[live], W)
+        l = log_sum_exp(z)
+        lse[live] = l
+        lp[live] = z[np.arange(live.size), targets[live]] - l
+    return lp, lse
+
+
+def sequence_sums(lp, logp_inf, mask, seq_id, S):
+    """Masked per-sequence sums.
+
+    s_i = sum_{n in seq i} m_n lp_n                (= ln pi(y_i | x), Eq. 3)
+    D_i = sum_{n in seq i} m_n (lp_n - logp_inf_n) (= ln pi/pi_vllm, Eq. 3)
+    T_i = sum_{n in seq i} m_n                     (response length)
+    """
+    m = np.asarray(mask).astype(np.float64)
+    seq_id = np.asarray(seq_id).astype(np.int64)
+    lp = np.asarray(lp, dtype=np.float64)
+    q = np.asarray(logp_inf, dtype=np.float64)
+    s = np.zeros(S)
+    D = np.zeros(S)
+    T = np.zeros(S)
+    # where(mask) keeps unread logp_inf entries (possibly NaN) out of the sums
+    diff = np.where(m > 0, lp - np.where(m > 0, q, 0.0), 0.0)
+    np.add.at(s, seq_id, m * lp)
+    np.add.at(D, seq_id, diff)
+    np.add.at(T, seq_id, m)
+    return s, D, T
+
+
+# --------------------------------------------------------------------------
+# Eq. 2: value estimate
+# --------------------------------------------------------------------------
+def value_estimate(reward, group_id, P, beta_v):
+    """V^_p = beta ln( (1/G_p) sum_{i in group p} exp(r_i / beta) )   (Eq. 2).
+
+    Evaluated in the algebraically identical max-shifted form so that small
+    beta does not overflow.  G_p is the actual member count; a group without
+    members gets 0.
+    """
+    r = np.asarray(reward, dtype=np.float64)
+    g = np.asarray(group_id).astype(np.int64)
+    vhat = np.zeros(P)
+    for p in range(P):
+        rp = r[g == p]
+        if rp.size == 0:
+            continue
+        R = rp.max()
+        vhat[p] = R + beta_v * np.log(np.mean(np.exp((rp - R) / beta_v)))
+    return vhat
+
+
+# --------------------------------------------------------------------------
+# Eq. 3: loss
+# --------------------------------------------------------------------------
+def loss_from_sums(D, reward, group_id, P, beta_v, beta_loss, loss_scale):
+    """Advantage, residual, loss and dL/ds_i from the per-sequence log-ratios.
+
+    A_i     = r_i - V^_{g(i)}                    (text below Eq. 2)
+    delta_i = beta_loss * D_i - A_i              (the bracket of Eq. 3)
+    L       = loss_scale * sum_i delta_i^2       (Eq. 3; loss_scale = 1 is the
+                                                  paper's plain double sum)
+    c_i     = dL/dD_i = 2 loss_scale beta_loss delta_i
+    """
+    r = np.asarray(reward, dtype=np.float64)
+    g = np.asarray(group_id).astype(np.int64)
+    vhat = value_estimate(r, g, P, beta_v)
+    A = r - vhat[g]
+    delta = beta_loss * np.asarray(D, dtype=np.float64) - A
+    loss = loss_scale * np.sum(delta * delta)
+    coef = 2.0 * loss_scale * beta_loss * delta
+    return dict(loss=loss, vhat=vhat, A=A, delta=delta, coef=coef)
+
+
+def loss_fwd(H, W, targets, mask, seq_id, group_id, reward, logp_inf,
+             S, P, beta_v, beta_loss, loss_scale):
+    """Whole forward: token log-probs -> sequence sums -> Eq. 2 -> Eq. 3."""
+    lp, lse = token_logprobs(H, W, targets, mask)
+    s, D, T = sequence_sums(lp, logp_inf, mask, seq_id, S)
+    out = loss_from_sums(D, reward, group_id, P, beta_v, beta_loss, loss_scale)
+    out.update(token_logp=lp, lse=lse, seq_logp=s, D=D, T=T)
+    return out
+
+
+# --------------------------------------------------------------------------
+# gradient of Eq. 3 with respect to H and W
+# --------------------------------------------------------------------------
+def loss_bwd(H, W, targets, mask, seq_id, coef):
+    """dL/dH [N, d] and dL/dW [V, d].
+
+    With p[n, v] = softmax_v z[n, v] and c_i = dL/ds_i, the chain rule through
+    s_i = sum_n m_n (z[n, y_n] - lse_n) gives
+        g[n, v] = dL/dz[n, v] = c_{seq(n)} m_n ( [v == y_n] - p[n, v] ),
+        dH = g . W,      dW = g^T . H.
+    Rows with mask == 0 have g = 0, hence a zero row in dH.
+    """
+    H = np.asarray(H, dtype=np.float64)
+    W = np.asarray(W, dtype=np.float64)
+    N, d = H.shape
+    mask = np.asarray(mask).astype(bool)
+    targets = np.asarray(targets).astype(np.int64)
+    seq_id = np.asarray(seq_id).astype(np.int64)
+    coef = np.asarray(coef, dtype=np.float64)
+    dH = np.zeros((N, d))
+    dW = np.zeros_like(W)
+    live = np.flatnonzero(mask)
+    if live.size == 0:
+        return dH, dW
+    z = logits(H[live], W)
+    l = log_sum_exp(z)
+    g = -np.exp(z - l[:, None])
+    g[np.arange(live.size), targets[live]] += 1.0
+    g *= coef[seq_id[live]][:, None]
+    dH[live] = g @ W
+    dW = g.T @ H[live]
+    return dH, dW
+
+
+def token_entropy(H, W, mask):
+    """Per-row policy entropy -sum_v p ln p (the diagnostic tracked in the
+    paper's entropy figure); 0 on masked rows."""
+    H = np.asarray(H, dtype=np.float64)
+    mask = np.asarray(mask).astype(bool)
+    ent = np.zeros(H.shape[0])
+    live = np.flatnonzero(mask)
+    if live.size:
+        z = logits(H[live], W)
+        l = log_sum_exp(z)
+        p = np.exp(z - l[:, None])
+        ent[live] = l - (p * z).sum(axis=1)
+    return ent
+
+
+# --------------------------------------------------------------------------
+# one-row / one-vocab-row forms for sampled checks at sizes where the whole
+# [N, V] problem is out of reach for a CPU.  Same definitions, one row each.
+# --------------------------------------------------------------------------
+def row_logprob(h, W, target):
+    """(lp, lse) for a single hidden-state row h [d]."""
+    z = np.asarray(W, dtype=np.float64) @ np.asarray(h, dtype=np.float64)
+    M = z.max()
+    lse = M + np.log(np.exp(z - M).sum())
+    return z[int(target)] - lse, lse
+
+
+def row_dH(h, W, target, c):
+    """dL/dh for a single live row with sequence coefficient c."""
+    W = np.asarray(W, dtype=np.float64)
+    z = W @ np.asarray(h, dtype=np.float64)
+    M = z.max()
+    lse = M + np.log(np.exp(z - M).sum())
+    g = -np.exp(z - lse)
+    g[int(target)] += 1.0
+    return c * (g @ W)
+
+
+def vocab_row_dW(v, w_v, H, targets, mask, seq_id, coef, lse):
+    """dL/dW[v, :] given every live row's log-sum-exp.
+
+    z[n, v] needs only row v of W, so one vocabulary row of dW costs O(N d).
+    """
+    H = np.asarray(H, dtype=np.float64)
+    m = np.asarray(mask).astype(np.float64)
+    z_v = H @ np.asarray(w_v, dtype=np.float64)
+    p_v = np.where(m > 0, np.exp(z_v - np.asarray(lse, dtype=np.float64)), 0.0)
+    onehot = (np.asarray(targets).astype(np.int64) == int(v)).astype(np.float64)
+    g_v = np.asarray(coef, dtype=np.float64)[np.asarray(seq_id).astype(np.int64)] * m * (onehot - p_v)
+    return g_v @ H

@@ -1,0 +1,313 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+
+None of these re-types the oracle's formulas with the same library call: each
+is a brute-force loop, a closed form, a limit the paper states, an invariant,
+a different library routine, or a finite difference.
+"""
+import decimal
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.special
+
+from oracle import oapl_oracle as orc
+
+RNG = np.random.default_rng(1234)
+
+
+def _tiny(N=7, d=5, V=11, S=3, seed=0):
+    r = np.random.default_rng(seed)
+    H = r.normal(size=(N, d))
+    W = r.normal(size=(V, d)) * 0.7
+    targets = r.integers(0, V, size=N)
+    mask = np.ones(N, dtype=np.uint8)
+    mask[2] = 0
+    seq_id = np.sort(r.integers(0, S, size=N))
+    return H, W, targets, mask, seq_id
+
+
+# ---------------------------------------------------------------- logits / lse
+def test_logits_match_explicit_loops():
+    H, W, targets, mask, _ = _tiny()
+    N, d = H.shape
+    V = W.shape[0]
+    lp, lse = orc.token_logprobs(H, W, targets, mask)
+    for n in range(N):
+        if not mask[n]:
+            assert lp[n] == 0.0 and lse[n] == 0.0
+            continue
+        z = [sum(H[n, k] * W[v, k] for k in range(d)) for v in range(V)]
+        tot = sum(math.exp(zv) for zv in z)          # naive, unshifted
+        assert lp[n] == pytest.approx(z[targets[n]] - math.log(tot), abs=1e-12)
+        assert lse[n] == pytest.approx(math.log(tot), abs=1e-12)
+
+
+def test_softmax_rows_sum_to_one():
+    H, W, _, _, _ = _tiny(N=4, V=13)
+    V = W.shape[0]
+    for n in range(H.shape[0]):
+        Hn = np.repeat(H[n:n + 1], V, axis=0)
+        lp, _ = orc.token_logprobs(Hn, W, np.arange(V), np.ones(V, dtype=np.uint8))
+        assert abs(np.exp(lp).sum() - 1.0) < 1e-12
+
+
+def test_zero_weight_gives_uniform():
+    H, W, targets, mask, _ = _tiny(V=17)
+    lp, lse = orc.token_logprobs(H, np.zeros_like(W), targets, mask)
+    live = mask.astype(bool)
+    assert np.allclose(lp[live], -math.log(17), atol=1e-14)
+    lp2, _ = orc.token_logprobs(np.zeros_like(H), W, targets, mask)
+    assert np.allclose(lp2[live], -math.log(17), atol=1e-14)
+
+
+def test_two_token_vocab_is_logistic():
+    r = np.random.default_rng(3)
+    H = r.normal(size=(6, 4))
+    W = r.normal(size=(2, 4))
+    t = r.integers(0, 2, size=6)
+    lp, _ = orc.token_logprobs(H, W, t, np.ones(6, dtype=np.uint8))
+    for n in range(6):
+        z = W @ H[n]
+        other = z[1 - t[n]] - z[t[n]]
+        assert lp[n] == pytest.approx(-math.log1p(math.exp(other)), abs=1e-13)
+
+
+def test_against_scipy_log_softmax_and_large_logits():
+    r = np.random.default_rng(5)
+    H = r.normal(size=(9, 8)) * 40.0          # logits of magnitude ~100: needs the max shift
+    W = r.normal(size=(33, 8))
+    t = r.integers(0, 33, size=9)
+    lp, lse = orc.token_logprobs(H, W, t, np.ones(9, dtype=np.uint8))
+    z = np.einsum("nk,vk->nv", H, W)
+    ref = scipy.special.log_softmax(z, axis=1)
+    assert np.allclose(lp, ref[np.arange(9), t], atol=1e-10)
+    assert np.allclose(lse, scipy.special.logsumexp(z, axis=1), atol=1e-10)
+    assert np.all(np.isfinite(lp))
+
+
+def test_bf16_widening_is_exact():
+    import torch
+    x = torch.randn(1000, dtype=torch.float32).to(torch.bfloat16)
+    bits = x.view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(orc.bf16_bits_to_f64(bits), x.to(torch.float64).numpy())
+
+
+def test_sequence_sums_by_loop_and_nan_in_masked_rows():
+    r = np.random.default_rng(7)
+    N, S = 40, 5
+    lp = r.normal(size=N)
+    q = r.normal(size=N)
+    mask = (r.random(N) < 0.7).astype(np.uint8)
+    q[mask == 0] = np.nan
+    seq_id = np.sort(r.integers(0, S, size=N))
+    s, D, T = orc.sequence_sums(lp, q, mask, seq_id, S)
+    for i in range(S):
+        idx = [n for n in range(N) if seq_id[n] == i and mask[n]]
+        assert s[i] == pytest.approx(sum(lp[n] for n in idx), abs=1e-12)
+        assert D[i] == pytest.approx(sum(lp[n] - q[n] for n in idx), abs=1e-12)
+        assert T[i] == len(idx)
+
+
+# ---------------------------------------------------------------- Eq. 2
+def test_value_equal_rewards_and_singleton():
+    v = orc.value_estimate([0.7] * 8 + [3.0], [0] * 8 + [1], 3, 0.37)
+    assert v[0] == pytest.approx(0.7, abs=1e-15)
+    assert v[1] == pytest.approx(3.0, abs=1e-15)
+    assert v[2] == 0.0                                    # empty group
+
+
+def test_value_limits_stated_by_the_paper():
+    r = RNG.random(8)
+    g = np.zeros(8, dtype=int)
+    assert orc.value_estimate(r, g, 1, 1e-4)[0] == pytest.approx(r.max(), abs=1e-3)
+    assert orc.value_estimate(r, g, 1, 1e7)[0] == pytest.approx(r.mean(), abs=1e-6)
+
+
+def test_value_binary_closed_form():
+    for beta in (0.1, 0.5, 1.0, 2.0, 10.0):
+        for k in range(0, 9):
+            r = np.array([1.0] * k + [0.0] * (8 - k))
+            want = beta * math.log(1.0 + (k / 8.0) * math.expm1(1.0 / beta))
+            got = orc.value_estimate(r, np.zeros(8, dtype=int), 1, beta)[0]
+            assert got == pytest.approx(want, rel=1e-12, abs=1e-13)
+
+
+def test_value_literal_formula_in_decimal_arithmetic():
+    decimal.getcontext().prec = 60
+    r = [0.0, 1.0, 1.0, 0.0, 0.25, 1.0, 0.0, 0.5]
+    for beta in (1e-3, 1e-2, 0.3, 1.0, 5.0):
+        tot = sum((decimal.Decimal(x) / decimal.Decimal(beta)).exp() for x in r)
+        want = float(decimal.Decimal(beta) * (tot / len(r)).ln())
+        got = orc.value_estimate(r, np.zeros(len(r), dtype=int), 1, beta)[0]
+        assert got == pytest.approx(want, rel=1e-12)
+
+
+def test_value_shift_bounds_monotone_and_scattered_groups():
+    r = RNG.normal(size=12)
+    g = np.array([0, 1, 2] * 4)                          # members not adjacent
+    v = orc.value_estimate(r, g, 3, 0.8)
+    v_shift = orc.value_estimate(r + 2.5, g, 3, 0.8)
+    assert np.allclose(v_shift, v + 2.5, atol=1e-13)
+    prev = None
+    for beta in (0.05, 0.2, 1.0, 4.0, 50.0):
+        vb = orc.value_estimate(r, g, 3, beta)
+        for p in range(3):
+            rp = r[g == p]
+            assert rp.mean() - 1e-12 <= vb[p] <= rp.max() + 1e-12
+        if prev is not None:
+            assert np.all(vb <= prev + 1e-12)            # non-increasing in beta
+        prev = vb
+
+
+# ---------------------------------------------------------------- Eq. 3
+def _problem(seed=0, N=24, d=6, V=19, S=6, P=2):
+    r = np.random.default_rng(seed)
+    H = r.normal(size=(N, d))
+    W = r.normal(size=(V, d)) * 0.5
+    targets = r.integers(0, V, size=N)
+    mask = (r.random(N) < 0.8).astype(np.uint8)
+    seq_id = np.sort(np.concatenate([np.arange(S), r.integers(0, S, size=N - S)]))
+    group_id = np.arange(S) % P
+    reward = (r.random(S) < 0.5).astype(np.float64)
+    logp_inf = r.normal(size=N) - 3.0
+    return dict(H=H, W=W, targets=targets, mask=mask, seq_id=seq_id, group_id=group_id,
+                reward=reward, logp_inf=logp_inf, S=S, P=P)
+
+
+def _fwd(p, beta_v=1.0, beta_loss=0.7, lam=1.0):
+    return orc.loss_fwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], p["group_id"],
+                        p["reward"], p["logp_inf"], p["S"], p["P"], beta_v, beta_loss, lam)
+
+
+def test_loss_is_the_literal_double_sum():
+    p = _problem()
+    beta_v, beta_loss = 1.3, 0.4
+    out = _fwd(p, beta_v, beta_loss, 1.0)
+    lp, _ = orc.token_logprobs(p["H"], p["W"], p["targets"], p["mask"])
+    total = 0.0
+    for x in range(p["P"]):
+        members = [i for i in range(p["S"]) if p["group_id"][i] == x]
+        vhat = beta_v * math.log(sum(math.exp(p["reward"][i] / beta_v) for i in members) / len(members))
+        for i in members:
+            rows = [n for n in range(len(lp)) if p["seq_id"][n] == i and p["mask"][n]]
+            ln_pi = sum(lp[n] for n in rows)
+            ln_pi_inf = sum(p["logp_inf"][n] for n in rows)
+            total += (beta_loss * (ln_pi - ln_pi_inf) - (p["reward"][i] - vhat)) ** 2
+    assert out["loss"] == pytest.approx(total, rel=1e-12)
+
+
+def test_zero_loss_and_zero_gradient_at_the_optimum():
+    # If beta ln(pi/pi_vllm) already equals r - V^ for every rollout, Eq. 3 is 0.
+    p = _problem(seed=2)
+    beta_v, beta_loss = 1.0, 0.5
+    first = _fwd(p, beta_v, beta_loss)
+    lp = first["token_logp"]
+    q = p["logp_inf"].copy()
+    for i in range(p["S"]):
+        rows = np.flatnonzero((p["seq_id"] == i) & (p["mask"] == 1))
+        assert rows.size > 0
+        want_D = first["A"][i] / beta_loss
+        q[rows] = lp[rows]
+        q[rows[0]] -= want_D
+    p["logp_inf"] = q
+    out = _fwd(p, beta_v, beta_loss)
+    assert out["loss"] < 1e-24
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    assert np.abs(dH).max() < 1e-10 and np.abs(dW).max() < 1e-10
+
+
+def test_loss_scalings():
+    p = _problem(seed=4)
+    a = _fwd(p, 1.0, 0.7, 1.0)["loss"]
+    b = _fwd(p, 1.0, 0.7, 1.0 / p["S"])["loss"]
+    assert b == pytest.approx(a / p["S"], rel=1e-13)
+    p["reward"][:] = 1.0                                   # A = 0: loss = lam * beta^2 * sum D^2
+    c = _fwd(p, 1.0, 0.7, 1.0)
+    d = _fwd(p, 1.0, 1.4, 1.0)
+    assert np.allclose(c["A"], 0.0, atol=1e-15)
+    assert d["loss"] == pytest.approx(4.0 * c["loss"], rel=1e-12)
+    assert c["loss"] == pytest.approx(0.49 * np.sum(c["D"] ** 2), rel=1e-12)
+
+
+def test_paper_hyperparameters_fixture():
+    path = os.path.join(os.path.dirname(__file__), "golden", "paper_hparams.txt")
+    kv = {}
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            k, *v = line.split()
+            kv[k] = v
+    beta_v, beta_loss, G = float(kv["beta_v"][0]), float(kv["beta_loss"][0]), int(kv["generations_per_prompt"][0])
+    assert (beta_v, beta_loss, G) == (1.0, 1e-3, 8)
+    # with those temperatures and k of 8 binary rewards correct
+    r = np.array([1, 0, 0, 1, 0, 0, 0, 1], dtype=float)
+    v = orc.value_estimate(r, np.zeros(8, dtype=int), 1, beta_v)[0]
+    assert v == pytest.approx(math.log(1 + 3 / 8 * (math.e - 1)), rel=1e-13)
+
+
+# ---------------------------------------------------------------- gradient
+def test_gradient_matches_central_differences():
+    p = _problem(seed=9, N=18, d=4, V=9, S=4, P=2)
+    beta_v, beta_loss, lam = 0.9, 0.6, 0.25
+    out = _fwd(p, beta_v, beta_loss, lam)
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    h = 1e-6
+    for name, grad in (("H", dH), ("W", dW)):
+        base = p[name]
+        for idx in np.ndindex(*base.shape):
+            q = dict(p)
+            plus, minus = base.copy(), base.copy()
+            plus[idx] += h
+            minus[idx] -= h
+            q[name] = plus
+            lp_ = _fwd(q, beta_v, beta_loss, lam)["loss"]
+            q[name] = minus
+            lm_ = _fwd(q, beta_v, beta_loss, lam)["loss"]
+            fd = (lp_ - lm_) / (2 * h)
+            assert grad[idx] == pytest.approx(fd, rel=2e-6, abs=2e-7), (name, idx)
+
+
+def test_gradient_invariants():
+    p = _problem(seed=11)
+    out = _fwd(p)
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    assert np.abs(dW.sum(axis=0)).max() < 1e-12          # rows of g sum to 0
+    assert np.all(dH[p["mask"] == 0] == 0.0)
+    dH0, _ = orc.loss_bwd(p["H"], np.zeros_like(p["W"]), p["targets"], p["mask"], p["seq_id"], out["coef"])
+    assert np.all(dH0 == 0.0)
+    never = [v for v in range(p["W"].shape[0]) if v not in set(p["targets"][p["mask"] == 1])]
+    z = p["H"] @ p["W"].T
+    prob = np.exp(z - out["lse"][:, None])
+    for v in never[:3]:
+        want = -sum(out["coef"][p["seq_id"][n]] * prob[n, v] * p["H"][n]
+                    for n in range(len(z)) if p["mask"][n])
+        assert np.allclose(dW[v], want, atol=1e-12)
+
+
+def test_sampled_forms_agree_with_full_forms():
+    p = _problem(seed=13)
+    out = _fwd(p)
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    for n in np.flatnonzero(p["mask"])[:5]:
+        lp, lse = orc.row_logprob(p["H"][n], p["W"], p["targets"][n])
+        assert lp == pytest.approx(out["token_logp"][n], abs=1e-12)
+        g = orc.row_dH(p["H"][n], p["W"], p["targets"][n], out["coef"][p["seq_id"][n]])
+        assert np.allclose(g, dH[n], atol=1e-12)
+    for v in (0, 5, 18):
+        row = orc.vocab_row_dW(v, p["W"][v], p["H"], p["targets"], p["mask"], p["seq_id"],
+                               out["coef"], out["lse"])
+        assert np.allclose(row, dW[v], atol=1e-12)
+
+
+def test_entropy_definition():
+    H, W, _, mask, _ = _tiny()
+    ent = orc.token_entropy(H, W, mask)
+    for n in range(H.shape[0]):
+        if not mask[n]:
+            assert ent[n] == 0.0
+            continue
+        z = W @ H[n]
+        pr = np.exp(z) / np.exp(z).sum()
+        assert ent[n] == pytest.approx(-(pr * np.log(pr)).sum(), abs=1e-12)
+    assert orc.token_entropy(H, np.zeros_like(W), mask)[0] == pytest.approx(math.log(W.shape[0]))
