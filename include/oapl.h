@@ -1,0 +1,148 @@
+/*
+ * oapl.h -- C ABI of the B200 (sm_100a) OAPL LM-head library.
+ *
+ * The library computes, for a batch of sampled responses, the trainer policy's
+ * sequence log-probabilities ln pi(y_i|x) through the LM head, the group value
+ * estimate of Eq. 2, the squared-regression objective of Eq. 3 of the OAPL paper
+ * ("Method" section), and the gradient of Eq. 3 with respect to the hidden states
+ * and the LM-head weight (Algorithm 1 takes gradient steps on Eq. 3), without ever
+ * forming the [N, V] logits tensor.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the parameter comment says "host".
+ *   - The caller owns every buffer.  The library allocates nothing, frees nothing
+ *     and never synchronises the device (oapl_get_last_status excepted); all work
+ *     is enqueued on `stream` (a cudaStream_t passed as void*).
+ *   - Return value: OAPL_OK (0) or a negative oapl_status.  On an argument error
+ *     nothing is enqueued.  Errors that only the device can see (a target outside
+ *     [0,V) on a live row, decreasing seq_id, a pipeline wait that gave up) are
+ *     recorded in the workspace and read back with oapl_get_last_status.
+ *   - The current CUDA device must be the one that owns the buffers.
+ */
+#ifndef OAPL_H_
+#define OAPL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  OAPL_OK = 0,
+  OAPL_ERR_INVALID_ARG = -1,         /* null pointer, non-positive size, beta <= 0 or not finite */
+  OAPL_ERR_MISALIGNED = -2,          /* H, W, dH, dW or workspace not 16-byte aligned */
+  OAPL_ERR_WORKSPACE_TOO_SMALL = -3, /* ws_bytes < oapl_workspace_bytes(problem, flags) */
+  OAPL_ERR_UNSUPPORTED_SHAPE = -4,   /* d not a multiple of 64, or sizes beyond int32 index range */
+  OAPL_ERR_BAD_TARGET = -5,          /* device: mask==1 and target outside [0,V) */
+  OAPL_ERR_BAD_SEQ_ORDER = -6,       /* device: seq_id decreasing or outside [0,S) */
+  OAPL_ERR_NONFINITE_INPUT = -7,     /* device: non-finite reward, or group_id outside [0,P) */
+  OAPL_ERR_DEVICE_TIMEOUT = -8,      /* device: a bounded pipeline wait expired */
+  OAPL_ERR_CUDA = -9,                /* a CUDA runtime/driver call failed */
+  OAPL_ERR_BAD_STATE = -10           /* oapl_loss_bwd without a matching oapl_loss_fwd in ws */
+} oapl_status;
+
+/* flags */
+#define OAPL_FLAG_NONE 0
+
+/*
+ * One batch, as the paper states the problem (Eq. 2 / Eq. 3): for every prompt x a
+ * group of rollouts y_i with rewards r(x, y_i) and the inference engine's
+ * log-probabilities; the trainer policy enters through the hidden states H and the
+ * LM-head weight W.  Row n of H predicts targets[n]; rows of one sequence are
+ * contiguous; only rows with mask==1 (response tokens) count in ln pi(y|x).
+ */
+typedef struct {
+  int64_t N;               /* row positions (padded or packed; the mask decides)             */
+  int32_t d;               /* hidden size, multiple of 64                                    */
+  int32_t V;               /* vocabulary size, >= 1                                          */
+  int32_t S;               /* sequences (rollouts)                                           */
+  int32_t P;               /* prompts (groups)                                               */
+  const void* H;           /* [N, d] bf16 row-major, 16-byte aligned                         */
+  const void* W;           /* [V, d] bf16 row-major, 16-byte aligned; logits = H . W^T       */
+  const int32_t* targets;  /* [N]; in [0,V) where mask==1; not read where mask==0            */
+  const uint8_t* mask;     /* [N]; 1 = response token                                        */
+  const int32_t* seq_id;   /* [N]; non-decreasing, in [0,S)                                  */
+  const int32_t* group_id; /* [S]; in [0,P); members of a group need not be adjacent         */
+  const float* reward;     /* [S]; finite                                                    */
+  const float* logp_inf;   /* [N]; inference-policy token log-probs; read only where mask==1 */
+  float beta_v;            /* temperature of Eq. 2 (the paper's beta_1), > 0                 */
+  float beta_loss;         /* temperature of Eq. 3 (the paper's beta_2), > 0                 */
+  float loss_scale;        /* lambda: 1 = Eq. 3's plain double sum; 1/S = mean per rollout   */
+} oapl_problem;
+
+/*
+ * Bytes of device workspace the calls below need for `problem` (host call; reads
+ * only N, d, V, S, P).  Returns 0 on invalid sizes.  The size grows with N*d and
+ * with V (a bounded row-chunk of bf16 logit gradients), never with N*V.
+ */
+size_t oapl_workspace_bytes(const oapl_problem* problem /*host*/, int flags);
+
+/*
+ * ln pi(y_t | x, y_<t) for every row and ln pi(y_i|x) for every sequence: the log
+ * of the policy's next-token distribution at the sampled token, summed over the
+ * response tokens (the quantity pi(y_i|x) that enters Eq. 3).
+ *   token_logp [N] f32: 0 where mask==0.       seq_logp [S] f32 or NULL.
+ * Reads H, W, targets, mask, seq_id of `problem`; the other fields may be null.
+ */
+int oapl_token_logprobs(const oapl_problem* problem /*host*/, float* token_logp, float* seq_logp,
+                        void* ws, size_t ws_bytes, int flags, void* stream);
+
+/*
+ * Eq. 2: vhat[p] = beta_v * ln( (1/G_p) * sum_{i in group p} exp(reward[i]/beta_v) ),
+ * evaluated in max-shifted form; G_p is the member count; a group without members
+ * gets 0.  reward [S], group_id [S], vhat [P].  No workspace.
+ */
+int oapl_value_estimate(const float* reward, const int32_t* group_id, int32_t S, int32_t P,
+                        float beta_v, float* vhat, void* stream);
+
+/*
+ * Eq. 3 forward: token log-probs -> masked per-sequence log-ratio D_i against
+ * logp_inf -> Eq. 2 -> advantage A_i = r_i - vhat -> residual
+ * delta_i = beta_loss*D_i - A_i -> loss = loss_scale * sum_i delta_i^2.
+ *   loss [1], seq_logp [S], vhat [P], delta [S] (may be NULL), token_logp [N] (may be NULL).
+ * Leaves in `ws` what oapl_loss_bwd needs (per-row log-sum-exp, per-sequence
+ * coefficients 2*loss_scale*beta_loss*delta_i).
+ */
+int oapl_loss_fwd(const oapl_problem* problem /*host*/, float* loss, float* seq_logp, float* vhat,
+                  float* delta, float* token_logp, void* ws, size_t ws_bytes, int flags, void* stream);
+
+/*
+ * Gradient of Eq. 3: with p = softmax(logits) and c_i the coefficient of the row's
+ * sequence, g[n,v] = c_i * mask_n * ([v == target_n] - p[n,v]);  dH = g . W,
+ * dW = g^T . H.  Must follow oapl_loss_fwd on the same problem and workspace.
+ *   dH [N, d] bf16 (rows with mask==0 are written as 0);
+ *   dW [V, d] f32; overwritten, or added to when accumulate_dW != 0.
+ */
+int oapl_loss_bwd(const oapl_problem* problem /*host*/, void* dH, float* dW, int accumulate_dW,
+                  void* ws, size_t ws_bytes, int flags, void* stream);
+
+/* Synchronises `stream` and returns the status word the device recorded in `ws`
+ * since the last forward call (OAPL_OK if none). */
+int oapl_get_last_status(void* ws, void* stream);
+
+/* Number of live rows (mask==1) counted by the last forward call on `ws`;
+ * synchronises `stream`.  Negative oapl_status on error. */
+int64_t oapl_get_live_rows(void* ws, void* stream);
+
+/* Kernel launches enqueued by this library in this process so far. */
+uint64_t oapl_launch_count(void);
+
+const char* oapl_status_string(int status);
+
+/*
+ * Bring-up aid for the tensor-core main loop shared by every contraction above:
+ * C[M, N] (f32 row-major, ld = N) = A . B with bf16 operands, through the same
+ * TMA/tcgen05 pipeline.  a_mn == 0: A is [M, K] row-major (K contiguous);
+ * a_mn == 1: A is stored [K, M] row-major (M contiguous).  b_mn == 0: B is stored
+ * [N, K] row-major; b_mn == 1: B is stored [K, N] row-major.  K % 64 == 0,
+ * M % 8 == 0, N % 8 == 0.  `err` is a device int the kernel sets on a timeout.
+ */
+int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn,
+                    int b_mn, int* err, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OAPL_H_ */

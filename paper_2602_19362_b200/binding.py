@@ -1,0 +1,172 @@
+"""ctypes binding of liboapl.so: same names as the C entry points, argument
+marshalling only.  Tensors are torch CUDA tensors used as device memory; every
+step of the path runs in the library's kernels.  There is no fallback: a missing
+library raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liboapl.so")
+
+OAPL_OK = 0
+STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL",
+          -4: "UNSUPPORTED_SHAPE", -5: "BAD_TARGET", -6: "BAD_SEQ_ORDER", -7: "NONFINITE_INPUT",
+          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE"}
+
+EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
+           "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
+           "oapl_status_string", "oapl_debug_gemm"]
+
+
+class OaplProblem(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int64), ("d", ctypes.c_int32), ("V", ctypes.c_int32),
+                ("S", ctypes.c_int32), ("P", ctypes.c_int32),
+                ("H", ctypes.c_void_p), ("W", ctypes.c_void_p), ("targets", ctypes.c_void_p),
+                ("mask", ctypes.c_void_p), ("seq_id", ctypes.c_void_p), ("group_id", ctypes.c_void_p),
+                ("reward", ctypes.c_void_p), ("logp_inf", ctypes.c_void_p),
+                ("beta_v", ctypes.c_float), ("beta_loss", ctypes.c_float), ("loss_scale", ctypes.c_float)]
+
+
+class OaplError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS.get(status, status)} ({lib().oapl_status_string(status).decode()})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load liboapl.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2602_19362_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+        pp = ctypes.POINTER(OaplProblem)
+        L.oapl_workspace_bytes.restype = sz
+        L.oapl_workspace_bytes.argtypes = [pp, i32]
+        L.oapl_token_logprobs.restype = i32
+        L.oapl_token_logprobs.argtypes = [pp, vp, vp, vp, sz, i32, vp]
+        L.oapl_value_estimate.restype = i32
+        L.oapl_value_estimate.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, f32, vp, vp]
+        L.oapl_loss_fwd.restype = i32
+        L.oapl_loss_fwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, i32, vp]
+        L.oapl_loss_bwd.restype = i32
+        L.oapl_loss_bwd.argtypes = [pp, vp, vp, i32, vp, sz, i32, vp]
+        L.oapl_get_last_status.restype = i32
+        L.oapl_get_last_status.argtypes = [vp, vp]
+        L.oapl_get_live_rows.restype = i64
+        L.oapl_get_live_rows.argtypes = [vp, vp]
+        L.oapl_launch_count.restype = ctypes.c_uint64
+        L.oapl_launch_count.argtypes = []
+        L.oapl_status_string.restype = ctypes.c_char_p
+        L.oapl_status_string.argtypes = [i32]
+        L.oapl_debug_gemm.restype = i32
+        L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check_dev(t, dtype, name):
+    if t is None:
+        return
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+
+
+def make_problem(batch: dict, beta_v=None, beta_loss=None, loss_scale=None) -> OaplProblem:
+    """Fill the C struct from a batch dict (see synth.make_batch).  The dict's
+    tensors must stay alive while the struct is in use."""
+    _check_dev(batch["H"], torch.bfloat16, "H")
+    _check_dev(batch["W"], torch.bfloat16, "W")
+    _check_dev(batch["targets"], torch.int32, "targets")
+    _check_dev(batch["mask"], torch.uint8, "mask")
+    _check_dev(batch["seq_id"], torch.int32, "seq_id")
+    _check_dev(batch.get("group_id"), torch.int32, "group_id")
+    _check_dev(batch.get("reward"), torch.float32, "reward")
+    _check_dev(batch.get("logp_inf"), torch.float32, "logp_inf")
+    p = OaplProblem()
+    p.N, p.d, p.V, p.S, p.P = batch["N"], batch["d"], batch["V"], batch["S"], batch["P"]
+    p.H, p.W = batch["H"].data_ptr(), batch["W"].data_ptr()
+    p.targets, p.mask, p.seq_id = batch["targets"].data_ptr(), batch["mask"].data_ptr(), batch["seq_id"].data_ptr()
+    for k in ("group_id", "reward", "logp_inf"):
+        t = batch.get(k)
+        setattr(p, k, None if t is None else t.data_ptr())
+    p.beta_v = batch.get("beta_v", 1.0) if beta_v is None else beta_v
+    p.beta_loss = batch.get("beta_loss", 1.0) if beta_loss is None else beta_loss
+    p.loss_scale = batch.get("loss_scale", 1.0) if loss_scale is None else loss_scale
+    return p
+
+
+def oapl_workspace_bytes(problem: OaplProblem, flags: int = 0) -> int:
+    return int(lib().oapl_workspace_bytes(ctypes.byref(problem), flags))
+
+
+def alloc_workspace(problem: OaplProblem, flags: int = 0, device="cuda") -> torch.Tensor:
+    n = oapl_workspace_bytes(problem, flags)
+    if n == 0:
+        raise OaplError(-1, "oapl_workspace_bytes")
+    ws = torch.empty(n + 1024, dtype=torch.uint8, device=device)
+    off = (-ws.data_ptr()) % 1024
+    return ws[off:off + n]
+
+
+def oapl_token_logprobs(problem, token_logp, seq_logp, ws, flags=0):
+    rc = lib().oapl_token_logprobs(ctypes.byref(problem), _ptr(token_logp), _ptr(seq_logp), _ptr(ws),
+                                   ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_token_logprobs")
+
+
+def oapl_value_estimate(reward, group_id, P, beta_v, vhat):
+    rc = lib().oapl_value_estimate(_ptr(reward), _ptr(group_id), reward.numel(), P, beta_v, _ptr(vhat), _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_value_estimate")
+
+
+def oapl_loss_fwd(problem, loss, seq_logp, vhat, delta, token_logp, ws, flags=0):
+    rc = lib().oapl_loss_fwd(ctypes.byref(problem), _ptr(loss), _ptr(seq_logp), _ptr(vhat), _ptr(delta),
+                             _ptr(token_logp), _ptr(ws), ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_loss_fwd")
+
+
+def oapl_loss_bwd(problem, dH, dW, accumulate_dW, ws, flags=0):
+    rc = lib().oapl_loss_bwd(ctypes.byref(problem), _ptr(dH), _ptr(dW), int(accumulate_dW), _ptr(ws),
+                             ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_loss_bwd")
+
+
+def oapl_get_last_status(ws) -> int:
+    return int(lib().oapl_get_last_status(_ptr(ws), _stream()))
+
+
+def oapl_get_live_rows(ws) -> int:
+    return int(lib().oapl_get_live_rows(_ptr(ws), _stream()))
+
+
+def oapl_launch_count() -> int:
+    return int(lib().oapl_launch_count())
+
+
+def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err):
+    rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), _ptr(err), _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_debug_gemm")

@@ -1,0 +1,387 @@
+// One persistent, warp-specialised tcgen05 contraction kernel, instantiated with
+// five epilogues:
+//   MODE_LSE   z = H.W^T tile by tile; per-row running (max, sum-exp) and target logit
+//   MODE_GRAD  z recomputed; g = c*(onehot - softmax) written as a bf16 row chunk
+//   MODE_DH    dH = g . W      (contraction over the vocabulary)
+//   MODE_DW    dW (+)= g^T . H (contraction over the rows of the chunk)
+//   MODE_DEBUG plain C = A.B for bring-up of the four operand-major combinations
+//
+// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM and issues the UMMAs,
+// warps 2..5 are the epilogue (one TMEM lane quadrant each).  Tile 128 x 256 x 64,
+// four shared-memory stages, two 256-column fp32 accumulators in TMEM so that the
+// epilogue of tile j overlaps the main loop of tile j+1.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "sm100_ptx.cuh"
+
+namespace oapl {
+
+enum { MODE_LSE = 0, MODE_GRAD = 1, MODE_DH = 2, MODE_DW = 3, MODE_DEBUG = 4 };
+
+constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;  // 16 KB
+constexpr int kBBytes = kBN * kBK * 2;  // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kErrTimeout = -8;  // OAPL_ERR_DEVICE_TIMEOUT
+
+struct GemmParams {
+  const int* n_live_ptr;  // device: number of live (compacted) rows; null in debug mode
+  int row_begin;          // first compacted row of this call's row range
+  int row_cap;            // capacity of the row range (whole problem, or one chunk)
+  int R, C;               // sweep schedule: R row blocks x C vocabulary splits per wave
+  int d, V;
+  int ldg;                // leading dimension of the g chunk (elements)
+  // MODE_LSE outputs: per (row, split) partials
+  float* pm;
+  float* pl;
+  float* pz;
+  // per compacted row
+  const int* tgt_c;
+  const int* seq_c;
+  const float* lse;
+  const float* coef;  // per sequence
+  __nv_bfloat16* G;   // chunk [row_cap, ldg]
+  const int* live_rows;
+  __nv_bfloat16* dH;  // [N, d]
+  float* dW;          // [V, d]
+  int accumulate;
+  // MODE_DEBUG
+  float* Cdbg;
+  int M, N, K;
+  int* err;  // device status word
+};
+
+struct Tile {
+  int m0, n0;    // tile origin (A's M coordinate, B's N coordinate)
+  int ka0, kb0;  // K origin for the A and B tensor maps
+  int nk;        // K steps of 64
+  int first, last, split;
+};
+
+template <int MODE>
+__device__ __forceinline__ bool get_tile(const GemmParams& p, int n_live, int j, Tile& t) {
+  t.first = t.last = 1;
+  t.split = 0;
+  if (MODE == MODE_LSE || MODE == MODE_GRAD) {
+    const int VT = (p.V + kBN - 1) / kBN;
+    const int rbi = blockIdx.x % p.R, s = blockIdx.x / p.R;
+    if (s >= p.C) return false;
+    const int vt0 = (int)((long long)VT * s / p.C), vt1 = (int)((long long)VT * (s + 1) / p.C);
+    const int per = vt1 - vt0;
+    if (per <= 0) return false;
+    const int wave = j / per, off = j - wave * per;
+    int row_end = p.row_begin + p.row_cap;
+    if (row_end > n_live) row_end = n_live;
+    const int rb = p.row_begin / kBM + wave * p.R + rbi;
+    if (rb * kBM >= row_end) return false;
+    t.m0 = rb * kBM;
+    t.n0 = (vt0 + off) * kBN;
+    t.ka0 = t.kb0 = 0;
+    t.nk = p.d / kBK;
+    t.first = (off == 0);
+    t.last = (off == per - 1);
+    t.split = s;
+    return true;
+  } else if (MODE == MODE_DH) {
+    int rows = n_live - p.row_begin;
+    if (rows > p.row_cap) rows = p.row_cap;
+    if (rows <= 0) return false;
+    const int MB = (rows + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
+    const int tix = blockIdx.x + j * gridDim.x;
+    if (tix >= MB * NB) return false;
+    t.m0 = (tix / NB) * kBM;  // row inside the chunk
+    t.n0 = (tix % NB) * kBN;
+    t.ka0 = t.kb0 = 0;
+    t.nk = (p.V + kBK - 1) / kBK;
+    return true;
+  } else if (MODE == MODE_DW) {
+    int rows = n_live - p.row_begin;
+    if (rows > p.row_cap) rows = p.row_cap;
+    if (rows <= 0) return false;
+    const int MB = (p.V + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
+    const int tix = blockIdx.x + j * gridDim.x;
+    if (tix >= MB * NB) return false;
+    t.m0 = (tix / NB) * kBM;  // vocabulary row
+    t.n0 = (tix % NB) * kBN;
+    t.ka0 = 0;            // g chunk rows are chunk-relative
+    t.kb0 = p.row_begin;  // compacted H rows are absolute
+    t.nk = (rows + kBK - 1) / kBK;
+    return true;
+  } else {
+    const int MB = (p.M + kBM - 1) / kBM, NB = (p.N + kBN - 1) / kBN;
+    const int tix = blockIdx.x + j * gridDim.x;
+    if (tix >= MB * NB) return false;
+    t.m0 = (tix / NB) * kBM;
+    t.n0 = (tix % NB) * kBN;
+    t.ka0 = t.kb0 = 0;
+    t.nk = p.K / kBK;
+    return true;
+  }
+}
+
+template <int MODE, int A_MN, int B_MN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
+  uint8_t* smem = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  const uint32_t bar0 = base + kStages * kStageBytes;
+  // barrier slots: full[0..3], empty[4..7], tmem_full[8..9], tmem_empty[10..11]
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_live = (MODE == MODE_DEBUG) ? 0 : *p.n_live_ptr;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 4);
+    }
+    *abort_flag = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+  }
+  if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      Tile t;
+      bool ok = true;
+      for (int j = 0; ok && get_tile<MODE>(p, n_live, j, t); ++j) {
+        for (int kb = 0; kb < t.nk; ++kb, ++it) {
+          const int s = it % kStages;
+          if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+            ok = false;
+            break;
+          }
+          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+          mbar_expect_tx(full_bar(s), kStageBytes);
+          const int ka = t.ka0 + kb * kBK, kbb = t.kb0 + kb * kBK;
+          if (A_MN) {
+#pragma unroll
+            for (int b = 0; b < kBM / 64; ++b)
+              tma_load_2d(sa + b * 8192, &tmA, full_bar(s), t.m0 + 64 * b, ka);
+          } else {
+            tma_load_2d(sa, &tmA, full_bar(s), ka, t.m0);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int b = 0; b < kBN / 64; ++b)
+              tma_load_2d(sb + b * 8192, &tmB, full_bar(s), t.n0 + 64 * b, kbb);
+          } else {
+            tma_load_2d(sb, &tmB, full_bar(s), kbb, t.n0);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, A_MN, B_MN);
+      uint32_t it = 0;
+      Tile t;
+      bool ok = true;
+      for (int j = 0; ok && get_tile<MODE>(p, n_live, j, t); ++j) {
+        const int buf = j & 1;
+        if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kBN;
+        for (int kb = 0; kb < t.nk; ++kb, ++it) {
+          const int s = it % kStages;
+          if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk) {
+            const uint64_t da = A_MN ? smem_desc_sw128(sa + kk * 2048, 8192, 1024)
+                                     : smem_desc_sw128(sa + kk * 32, 16, 1024);
+            const uint64_t db = B_MN ? smem_desc_sw128(sb + kk * 2048, 8192, 1024)
+                                     : smem_desc_sw128(sb + kk * 32, 16, 1024);
+            umma_bf16(d_tmem, da, db, idesc, (kb | kk) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(s));  // stage reusable once these UMMAs have read it
+        }
+        if (ok) umma_commit(tfull_bar(buf));  // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32)
+    const int r_in_tile = quad * 32 + lane;
+    // MODE_LSE running state of this thread's row (log2 domain for the max)
+    float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f;
+    Tile t;
+    for (int j = 0; get_tile<MODE>(p, n_live, j, t); ++j) {
+      const int buf = j & 1;
+      // per-row constants
+      const int row = t.m0 + r_in_tile;  // MODE_LSE/GRAD: compacted row; DH: chunk row; DW: vocab row
+      int tgt = -1;
+      float cf = 0.f, lse2 = 0.f;
+      bool valid = true;
+      if (MODE == MODE_LSE) {
+        valid = row < n_live;
+        tgt = valid ? p.tgt_c[row] : -1;
+        if (t.first) { run_m2 = -INFINITY; run_l = 0.f; run_z = 0.f; }
+      } else if (MODE == MODE_GRAD) {
+        valid = row < n_live;
+        if (valid) {
+          tgt = p.tgt_c[row];
+          cf = p.coef[p.seq_c[row]];
+          lse2 = p.lse[row] * kLog2e;
+        }
+      }
+      if (!mbar_wait(tfull_bar(buf), (j >> 1) & 1u, abort_flag)) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;
+#pragma unroll 1
+      for (int c = 0; c < kBN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c * 32, r);
+        tmem_ld_wait();
+        const int col0 = t.n0 + c * 32;
+        if (MODE == MODE_LSE) {
+          if (col0 < p.V) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+            if (col0 + 32 > p.V) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (col0 + i >= p.V) v[i] = -INFINITY;
+            }
+            float cmax = v[0];
+#pragma unroll
+            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+            const float m2 = fmaxf(run_m2, cmax * kLog2e);
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc += ex2_approx(fmaf(v[i], kLog2e, -m2));
+            run_l = run_l * ex2_approx(run_m2 - m2) + acc;
+            run_m2 = m2;
+            const int ti = tgt - col0;
+            if (ti >= 0 && ti < 32) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i == ti) run_z = v[i];
+            }
+          }
+        } else if (MODE == MODE_GRAD) {
+          uint32_t o[16];
+          if (valid && col0 < p.V) {
+            const int ti = tgt - col0;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              float g0 = -cf * ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -lse2));
+              float g1 = -cf * ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -lse2));
+              if (i == ti) g0 += cf;
+              if (i + 1 == ti) g1 += cf;
+              if (col0 + i >= p.V) g0 = 0.f;
+              if (col0 + i + 1 >= p.V) g1 = 0.f;
+              o[i >> 1] = pack_bf16x2(g0, g1);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = 0u;
+          }
+          if (col0 < p.ldg) {
+            uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)(row - p.row_begin) * p.ldg + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          }
+        } else if (MODE == MODE_DH) {
+          const int crow = p.row_begin + row;
+          if (crow < n_live && row < p.row_cap && col0 < p.d) {
+            uint32_t o[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+              o[i >> 1] = pack_bf16x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            uint4* dst = reinterpret_cast<uint4*>(p.dH + (size_t)p.live_rows[crow] * p.d + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          }
+        } else if (MODE == MODE_DW) {
+          if (row < p.V && col0 < p.d) {
+            float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)row * p.d + col0);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              float4 x = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                     __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+              if (p.accumulate) {
+                const float4 y = dst[q];
+                x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+              }
+              dst[q] = x;
+            }
+          }
+        } else {
+          if (row < p.M) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i < p.N) p.Cdbg[(size_t)row * p.N + col0 + i] = __uint_as_float(r[i]);
+          }
+        }
+      }
+      // accumulator drained: hand the TMEM buffer back to the UMMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (MODE == MODE_LSE) {
+        if (t.last && valid) {
+          const size_t o = (size_t)row * p.C + t.split;
+          p.pm[o] = run_m2 * 0.6931471805599453f;  // back to natural units
+          p.pl[o] = run_l;
+          p.pz[o] = run_z;
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) {
+      if (p.err) atomicCAS(p.err, 0, kErrTimeout);
+      const long long t0 = clock64();  // let loads already in flight land before smem is released
+      while (clock64() - t0 < 2000000LL) {
+      }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace oapl

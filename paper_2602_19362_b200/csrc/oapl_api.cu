@@ -1,0 +1,443 @@
+// Host side of the C ABI declared in include/oapl.h: argument validation, the
+// workspace carve-up, tensor-map encoding and the launch sequences.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "../../include/oapl.h"
+#include "gemm_sm100.cuh"
+#include "small_kernels.cuh"
+
+namespace oapl {
+
+static std::atomic<uint64_t> g_launches{0};
+#define OAPL_LAUNCHED() (g_launches.fetch_add(1, std::memory_order_relaxed))
+
+constexpr int kMaxSplits = 16;
+constexpr int kChunkRowsDefault = 74 * 128;  // half of a 148-SM wave of row blocks
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carve {
+  size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, pm, pl, pz, cstart,
+      cend, seq_D, coef, vhat, seq_logp, Hc, G, total;
+  int n_pad, nblk, chunk_rows, ldg;
+};
+
+static int env_int(const char* name, int dflt) {
+  const char* s = getenv(name);
+  return (s && *s) ? atoi(s) : dflt;
+}
+
+static bool carve(const oapl_problem* p, Carve* c) {
+  if (!p || p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return false;
+  if (p->d % 64 != 0) return false;
+  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000) return false;
+  const size_t n_pad = align_up((size_t)p->N, 128);
+  c->n_pad = (int)n_pad;
+  c->nblk = (int)((p->N + kScanBlock - 1) / kScanBlock);
+  int chunk = env_int("OAPL_CHUNK_ROWS", kChunkRowsDefault);
+  chunk = (int)align_up((size_t)(chunk < 128 ? 128 : chunk), 128);
+  if ((size_t)chunk > n_pad) chunk = (int)n_pad;
+  c->chunk_rows = chunk;
+  c->ldg = (int)align_up((size_t)p->V, 256);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 1024);
+    return o;
+  };
+  c->state = take(sizeof(DevState));
+  c->block_cnt = take(4 * (size_t)c->nblk);
+  c->block_off = take(4 * (size_t)c->nblk);
+  c->live_rows = take(4 * n_pad);
+  c->tgt_c = take(4 * n_pad);
+  c->seq_c = take(4 * n_pad);
+  c->q_c = take(4 * n_pad);
+  c->lp_c = take(4 * n_pad);
+  c->lse = take(4 * n_pad);
+  c->pm = take(4 * n_pad * kMaxSplits);
+  c->pl = take(4 * n_pad * kMaxSplits);
+  c->pz = take(4 * n_pad * kMaxSplits);
+  c->cstart = take(4 * (size_t)p->S);
+  c->cend = take(4 * (size_t)p->S);
+  c->seq_D = take(4 * (size_t)p->S);
+  c->coef = take(4 * (size_t)p->S);
+  c->vhat = take(4 * (size_t)p->P);
+  c->seq_logp = take(4 * (size_t)p->S);
+  c->Hc = take(2 * n_pad * (size_t)p->d);
+  c->G = take(2 * (size_t)chunk * (size_t)c->ldg);
+  c->total = off;
+  return true;
+}
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] row-major with leading dimension ld (elements); the box
+// is box_cols (= 64 elements = one 128-byte swizzle row) by box_rows.
+static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                     uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
+  }
+  return n;
+}
+
+// Sweep schedule: C vocabulary splits x R row blocks per wave, R*C <= SM count.  C is
+// the smallest power of two that keeps the wave's H row blocks within an L2 budget and
+// does not leave SMs without a row block when the row range is short.
+static void pick_sweep(int n_sm, int d, int rb_max, int vtiles, int* R, int* C) {
+  int c = env_int("OAPL_SPLITS", 0);
+  if (c <= 0) {
+    c = 1;
+    const size_t budget = (size_t)env_int("OAPL_L2_BUDGET_MB", 40) << 20;
+    while (c < kMaxSplits && (size_t)(n_sm / c) * 128 * d * 2 > budget) c *= 2;
+    while (c < kMaxSplits && n_sm / c > rb_max) c *= 2;
+  }
+  if (c > kMaxSplits) c = kMaxSplits;
+  while (c > 1 && c > vtiles) c /= 2;
+  int r = n_sm / c;
+  if (r < 1) r = 1;
+  if (r > rb_max) r = rb_max;
+  *R = r;
+  *C = c;
+}
+
+template <int MODE, int A_MN, int B_MN>
+static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& gp, int grid,
+                       cudaStream_t st) {
+  static bool attr_set = false;
+  auto kern = gemm_kernel<MODE, A_MN, B_MN>;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kGemmSmemBytes) != cudaSuccess)
+      return OAPL_ERR_CUDA;
+    attr_set = true;
+  }
+  kern<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(a, b, gp);
+  OAPL_LAUNCHED();
+  return cudaGetLastError() == cudaSuccess ? OAPL_OK : OAPL_ERR_CUDA;
+}
+
+static int check_problem(const oapl_problem* p, bool need_loss_inputs) {
+  if (!p) return OAPL_ERR_INVALID_ARG;
+  if (p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return OAPL_ERR_INVALID_ARG;
+  if (p->d % 64 != 0) return OAPL_ERR_UNSUPPORTED_SHAPE;
+  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000)
+    return OAPL_ERR_UNSUPPORTED_SHAPE;
+  if (!p->H || !p->W || !p->targets || !p->mask || !p->seq_id) return OAPL_ERR_INVALID_ARG;
+  if (((uintptr_t)p->H | (uintptr_t)p->W) & 15) return OAPL_ERR_MISALIGNED;
+  if (need_loss_inputs) {
+    if (!p->group_id || !p->reward || !p->logp_inf) return OAPL_ERR_INVALID_ARG;
+    if (!(p->beta_v > 0.f) || !std::isfinite(p->beta_v)) return OAPL_ERR_INVALID_ARG;
+    if (!(p->beta_loss > 0.f) || !std::isfinite(p->beta_loss)) return OAPL_ERR_INVALID_ARG;
+    if (!std::isfinite(p->loss_scale)) return OAPL_ERR_INVALID_ARG;
+  }
+  return OAPL_OK;
+}
+
+#define CK(call)                                   \
+  do {                                             \
+    if ((call) != cudaSuccess) return OAPL_ERR_CUDA; \
+  } while (0)
+#define CKL()                                                  \
+  do {                                                         \
+    OAPL_LAUNCHED();                                           \
+    if (cudaGetLastError() != cudaSuccess) return OAPL_ERR_CUDA; \
+  } while (0)
+
+// Shared forward: compaction, fused logits + online log-sum-exp, merge, per-sequence sums.
+static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, float* token_logp,
+                          float* seq_logp, bool with_q, cudaStream_t st) {
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  DevState* state = reinterpret_cast<DevState*>(ws + c.state);
+  int* block_cnt = reinterpret_cast<int*>(ws + c.block_cnt);
+  int* block_off = reinterpret_cast<int*>(ws + c.block_off);
+  int* live_rows = reinterpret_cast<int*>(ws + c.live_rows);
+  int* tgt_c = reinterpret_cast<int*>(ws + c.tgt_c);
+  int* seq_c = reinterpret_cast<int*>(ws + c.seq_c);
+  float* q_c = reinterpret_cast<float*>(ws + c.q_c);
+  float* lp_c = reinterpret_cast<float*>(ws + c.lp_c);
+  float* lse = reinterpret_cast<float*>(ws + c.lse);
+  int* cstart = reinterpret_cast<int*>(ws + c.cstart);
+  int* cend = reinterpret_cast<int*>(ws + c.cend);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + c.Hc);
+
+  CK(cudaMemsetAsync(state, 0, sizeof(DevState), st));
+  CK(cudaMemsetAsync(cstart, 0, 4 * (size_t)p->S, st));
+  CK(cudaMemsetAsync(cend, 0, 4 * (size_t)p->S, st));
+  if (token_logp) CK(cudaMemsetAsync(token_logp, 0, 4 * (size_t)p->N, st));
+
+  count_live_kernel<<<c.nblk, kScanBlock, 0, st>>>(p->mask, p->seq_id, p->targets, p->N, p->S, p->V,
+                                                   block_cnt, &state->status);
+  CKL();
+  scan_blocks_kernel<<<1, 1024, 0, st>>>(block_cnt, c.nblk, block_off, state);
+  CKL();
+  write_live_kernel<<<c.nblk, kScanBlock, 0, st>>>(p->mask, p->seq_id, p->targets,
+                                                   with_q ? p->logp_inf : nullptr, p->N, block_off,
+                                                   live_rows, tgt_c, seq_c, q_c);
+  CKL();
+  seq_bounds_kernel<<<n_sm * 2, 256, 0, st>>>(seq_c, state, cstart, cend);
+  CKL();
+  gather_rows_kernel<<<n_sm * 8, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(p->H), live_rows,
+                                               state, p->d, Hc);
+  CKL();
+
+  CUtensorMap tmA, tmB;
+  if (!make_map(&tmA, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128)) return OAPL_ERR_CUDA;
+  if (!make_map(&tmB, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256)) return OAPL_ERR_CUDA;
+  GemmParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.n_live_ptr = &state->n_live;
+  gp.row_begin = 0;
+  gp.row_cap = c.n_pad;
+  pick_sweep(n_sm, p->d, c.n_pad / 128, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+  gp.d = p->d;
+  gp.V = p->V;
+  gp.pm = reinterpret_cast<float*>(ws + c.pm);
+  gp.pl = reinterpret_cast<float*>(ws + c.pl);
+  gp.pz = reinterpret_cast<float*>(ws + c.pz);
+  gp.tgt_c = tgt_c;
+  gp.err = &state->status;
+  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, gp, gp.R * gp.C, st);
+  if (rc != OAPL_OK) return rc;
+
+  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.C, state, live_rows, lse, lp_c,
+                                             token_logp);
+  CKL();
+  seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp,
+                                        reinterpret_cast<float*>(ws + c.seq_D), with_q ? 1 : 0);
+  CKL();
+  return OAPL_OK;
+}
+
+}  // namespace oapl
+
+using namespace oapl;
+
+extern "C" {
+
+size_t oapl_workspace_bytes(const oapl_problem* problem, int /*flags*/) {
+  Carve c;
+  if (!carve(problem, &c)) return 0;
+  return c.total;
+}
+
+const char* oapl_status_string(int status) {
+  switch (status) {
+    case OAPL_OK: return "ok";
+    case OAPL_ERR_INVALID_ARG: return "invalid argument";
+    case OAPL_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case OAPL_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case OAPL_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (d must be a multiple of 64)";
+    case OAPL_ERR_BAD_TARGET: return "target outside [0,V) on a live row";
+    case OAPL_ERR_BAD_SEQ_ORDER: return "seq_id decreasing or outside [0,S)";
+    case OAPL_ERR_NONFINITE_INPUT: return "non-finite reward or group_id outside [0,P)";
+    case OAPL_ERR_DEVICE_TIMEOUT: return "device pipeline wait timed out";
+    case OAPL_ERR_CUDA: return "CUDA call failed";
+    case OAPL_ERR_BAD_STATE: return "backward called without a matching forward";
+    default: return "unknown status";
+  }
+}
+
+uint64_t oapl_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int oapl_get_last_status(void* ws, void* stream) {
+  if (!ws) return OAPL_ERR_INVALID_ARG;
+  Carve dummy;
+  (void)dummy;
+  DevState h;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return OAPL_ERR_CUDA;
+  return h.status;
+}
+
+int64_t oapl_get_live_rows(void* ws, void* stream) {
+  if (!ws) return OAPL_ERR_INVALID_ARG;
+  DevState h;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return OAPL_ERR_CUDA;
+  return h.n_live;
+}
+
+int oapl_value_estimate(const float* reward, const int32_t* group_id, int32_t S, int32_t P,
+                        float beta_v, float* vhat, void* stream) {
+  if (!reward || !group_id || !vhat || S <= 0 || P <= 0) return OAPL_ERR_INVALID_ARG;
+  if (!(beta_v > 0.f) || !std::isfinite(beta_v)) return OAPL_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  value_estimate_kernel<<<(P + 7) / 8, 256, 0, st>>>(reward, group_id, S, P, beta_v, vhat, nullptr);
+  CKL();
+  return OAPL_OK;
+}
+
+int oapl_token_logprobs(const oapl_problem* p, float* token_logp, float* seq_logp, void* ws,
+                        size_t ws_bytes, int /*flags*/, void* stream) {
+  int rc = check_problem(p, false);
+  if (rc != OAPL_OK) return rc;
+  if (!token_logp || !ws) return OAPL_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  return forward_common(p, c, static_cast<uint8_t*>(ws), token_logp, seq_logp, false,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int oapl_loss_fwd(const oapl_problem* p, float* loss, float* seq_logp, float* vhat, float* delta,
+                  float* token_logp, void* ws, size_t ws_bytes, int /*flags*/, void* stream) {
+  int rc = check_problem(p, true);
+  if (rc != OAPL_OK) return rc;
+  if (!loss || !seq_logp || !vhat || !ws) return OAPL_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = forward_common(p, c, w, token_logp, seq_logp, true, st);
+  if (rc != OAPL_OK) return rc;
+  DevState* state = reinterpret_cast<DevState*>(w + c.state);
+  value_estimate_kernel<<<(p->P + 7) / 8, 256, 0, st>>>(p->reward, p->group_id, p->S, p->P, p->beta_v,
+                                                        vhat, &state->status);
+  CKL();
+  loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, reinterpret_cast<float*>(w + c.seq_D),
+                                 p->S, p->P, p->beta_loss, p->loss_scale,
+                                 reinterpret_cast<float*>(w + c.coef), delta, loss, state);
+  CKL();
+  return OAPL_OK;
+}
+
+int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW, void* ws,
+                  size_t ws_bytes, int /*flags*/, void* stream) {
+  int rc = check_problem(p, true);
+  if (rc != OAPL_OK) return rc;
+  if (!dH || !dW || !ws) return OAPL_ERR_INVALID_ARG;
+  if (((uintptr_t)dH | (uintptr_t)dW) & 15) return OAPL_ERR_MISALIGNED;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DevState* state = reinterpret_cast<DevState*>(w + c.state);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(w + c.Hc);
+  __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(w + c.G);
+
+  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH));
+  CKL();
+  if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
+
+  CUtensorMap tmH, tmW, tmGk, tmWmn, tmGmn, tmHmn;
+  const uint64_t ldg = (uint64_t)c.ldg;
+  bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
+            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256) &&
+            make_map(&tmGk, G, (uint64_t)c.chunk_rows, ldg, ldg, 128) &&
+            make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
+            make_map(&tmGmn, G, (uint64_t)c.chunk_rows, ldg, ldg, 64) &&
+            make_map(&tmHmn, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 64);
+  if (!ok) return OAPL_ERR_CUDA;
+
+  GemmParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.n_live_ptr = &state->n_live;
+  gp.row_cap = c.chunk_rows;
+  gp.d = p->d;
+  gp.V = p->V;
+  gp.ldg = c.ldg;
+  gp.tgt_c = reinterpret_cast<int*>(w + c.tgt_c);
+  gp.seq_c = reinterpret_cast<int*>(w + c.seq_c);
+  gp.lse = reinterpret_cast<float*>(w + c.lse);
+  gp.coef = reinterpret_cast<float*>(w + c.coef);
+  gp.G = G;
+  gp.live_rows = reinterpret_cast<int*>(w + c.live_rows);
+  gp.dH = static_cast<__nv_bfloat16*>(dH);
+  gp.dW = dW;
+  gp.accumulate = 1;  // dW is zeroed above unless the caller accumulates; every chunk adds
+  gp.err = &state->status;
+  pick_sweep(n_sm, p->d, c.chunk_rows / 128, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+
+  // Row chunks of the compacted rows.  The live-row count lives on the device, so the
+  // host enqueues every chunk the row count N could need; chunks past the live rows
+  // find no tile and return at once.
+  for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
+    gp.row_begin = r0;
+    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, gp, gp.R * gp.C, st);
+    if (rc != OAPL_OK) return rc;
+    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, gp, n_sm, st);
+    if (rc != OAPL_OK) return rc;
+    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, gp, n_sm, st);
+    if (rc != OAPL_OK) return rc;
+  }
+  return OAPL_OK;
+}
+
+int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn, int b_mn,
+                    int* err, void* stream) {
+  if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return OAPL_ERR_INVALID_ARG;
+  if (K % 64 || M % 8 || N % 8) return OAPL_ERR_UNSUPPORTED_SHAPE;
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  CUtensorMap ta, tb;
+  bool ok = a_mn ? make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)M, 64)
+                 : make_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128);
+  ok = ok && (b_mn ? make_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)N, 64)
+                   : make_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, 256));
+  if (!ok) return OAPL_ERR_CUDA;
+  GemmParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.Cdbg = C;
+  gp.M = M;
+  gp.N = N;
+  gp.K = K;
+  gp.err = err;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+  const int grid = tiles < n_sm ? tiles : n_sm;
+  if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0>(ta, tb, gp, grid, st);
+  if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1>(ta, tb, gp, grid, st);
+  if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0>(ta, tb, gp, grid, st);
+  return launch_gemm<MODE_DEBUG, 1, 1>(ta, tb, gp, grid, st);
+}
+
+}  // extern "C"
