@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the OAPL LM-head hot path (loss forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl reference]
+
+A step is one oapl_loss_fwd + oapl_loss_bwd over one synthetic batch shaped like the
+paper's 7B-scale trainer step (d=3584, V=152064, 16 prompts x 8 rollouts, response
+lengths U[512,4096], padded layout).  The metric is response tokens per second; the
+roofline object credits 6*N*d*V flops per step against the measured dense-bf16 peak.
+Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "response tokens/sec for OAPL loss fwd+bwd"
+UNIT = "tokens/s"
+
+
+# ---------------------------------------------------------------------------- helpers
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(burst=float(p["bf16_tflops"]), sustained=float(p["bf16_tflops_sustained"]),
+                    hbm=float(p["hbm_gbs"]), source="measured")
+    return dict(burst=1590.0, sustained=1400.0, hbm=6650.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def reduce_max(value: float, dist, device) -> float:
+    """Max over ranks of a per-rank time (identity when not distributed)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def reduce_sum(value: float, dist, device) -> float:
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+# ---------------------------------------------------------------------------- oracle arm
+def oracle_sample(workload: str, live_rows: int):
+    """A bounded sample of the workload for the CPU oracle: same d, V, distributions and
+    betas, 2 prompts x 4 rollouts and about `live_rows` response tokens."""
+    import numpy as np
+    from oracle import oapl_oracle as orc
+    from paper_2602_19362_b200 import synth
+    wl = synth.small_variant(workload, prompts=2, samples=4, live_rows=live_rows) \
+        if workload != "tiny" else synth.WORKLOADS["tiny"]
+    b = synth.make_batch(wl, seed=0)
+    npy = lambda t: t.numpy()
+    args = dict(Hb=synth.bf16_bits(b["H"]), Wb=synth.bf16_bits(b["W"]), t=npy(b["targets"]),
+                m=npy(b["mask"]), s=npy(b["seq_id"]), g=npy(b["group_id"]), r=npy(b["reward"]),
+                q=npy(b["logp_inf"]))
+
+    def step():
+        Hd, Wd = orc.bf16_bits_to_f64(args["Hb"]), orc.bf16_bits_to_f64(args["Wb"])
+        f = orc.loss_fwd(Hd, Wd, args["t"], args["m"], args["s"], args["g"], args["r"], args["q"],
+                         b["S"], b["P"], b["beta_v"], b["beta_loss"], b["loss_scale"])
+        orc.loss_bwd(Hd, Wd, args["t"], args["m"], args["s"], f["coef"])
+        return f["loss"]
+
+    desc = (f"{wl.name}: {b['live_tokens']} response tokens in {b['S']} sequences, d={wl.d}, V={wl.V}, "
+            f"oracle loss fwd+bwd in fp64 numpy")
+    return step, b["live_tokens"], desc
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy  # noqa: F401  (loads BLAS before the thread count is read)
+    step, tokens, desc = oracle_sample(args.workload, args.ref_rows)
+    for _ in range(min(args.warmup, 1)):
+        step()
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    val = tokens / dt
+    cores = host_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": args.workload, "sample": desc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------- CUDA arm
+def run_cuda(args) -> None:
+    import torch
+    import torch.distributed as dist
+    from paper_2602_19362_b200 import binding as B, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    # cpu_baseline first (rank 0, N=1 only), before the device is busy
+    cpu_base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        step, tokens, desc = oracle_sample(args.workload, args.ref_rows)
+        t0 = time.perf_counter()
+        step()
+        dt = time.perf_counter() - t0
+        cpu_base = {"value": tokens / dt, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                    "sample": desc, "seconds": dt}
+
+    wl = synth.WORKLOADS[args.workload]
+    # data-parallel over prompts: every rank holds its own groups (weak scaling), W replicated
+    batch = synth.make_batch(wl, seed=args.seed + rank, device=str(dev), beta=args.beta)
+    N, S, P, d, V = (batch[k] for k in ("N", "S", "P", "d", "V"))
+    n_live = batch["live_tokens"]
+    prob = B.make_problem(batch)
+    ws = B.alloc_workspace(prob, device=dev)
+    loss = torch.zeros(1, device=dev)
+    seq_logp = torch.zeros(S, device=dev)
+    vhat = torch.zeros(P, device=dev)
+    delta = torch.zeros(S, device=dev)
+    dH = torch.empty(N, d, dtype=torch.bfloat16, device=dev)
+    dW = torch.empty(V, d, dtype=torch.float32, device=dev)
+
+    def step():
+        B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
+        B.oapl_loss_bwd(prob, dH, dW, False, ws)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st = B.oapl_get_last_status(ws)
+    if st != 0:
+        raise RuntimeError(f"device status {B.STATUS.get(st, st)}")
+    assert B.oapl_get_live_rows(ws) == n_live
+
+    # ---- timed region: device-resident inputs
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    B.oapl_profile_enable(True)
+    launches0 = B.oapl_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for k in range(args.steps):
+        B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
+        ev[2 * k + 1].record()
+        B.oapl_loss_bwd(prob, dH, dW, False, ws)
+        ev[2 * k + 2].record()
+    barrier()
+    launches = B.oapl_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[2 * args.steps])
+    fwd_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
+    bwd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
+    prof = B.oapl_profile_read()
+    B.oapl_profile_enable(False)
+    clocks = sampler.stop() if rank == 0 else None
+    st = B.oapl_get_last_status(ws)
+    if st != 0:
+        raise RuntimeError(f"device status {B.STATUS.get(st, st)}")
+    loss_val = float(loss.item())
+
+    ms_step = reduce_max(total_ms / args.steps, dist if world > 1 else None, dev)
+    tokens_all = reduce_sum(float(n_live), dist if world > 1 else None, dev)
+    value = tokens_all / (ms_step * 1e-3)
+
+    # ---- end to end: host-resident inputs and results, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        names = ["H", "targets", "mask", "seq_id", "group_id", "reward", "logp_inf"]
+        host_in = {k: batch[k].cpu().pin_memory() for k in names}
+        host_out = {"loss": torch.empty(1).pin_memory(), "seq_logp": torch.empty(S).pin_memory(),
+                    "dH": torch.empty(N, d, dtype=torch.bfloat16).pin_memory(),
+                    "dW": torch.empty(V, d, dtype=torch.float32).pin_memory()}
+        dev_out = {"loss": loss, "seq_logp": seq_logp, "dH": dH, "dW": dW}
+        h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+        d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+
+        def e2e_step():
+            for k in names:
+                batch[k].copy_(host_in[k], non_blocking=True)
+            step()
+            for k, t in host_out.items():
+                t.copy_(dev_out[k], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = reduce_max(e0.elapsed_time(e1) / n_e2e, dist if world > 1 else None, dev)
+        e2e = {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops_step = 6.0 * n_live * d * V          # credited: logits, dH, dW
+    gemm_ms = sum(v[0] for v in prof.values()) / args.steps
+    gemm_launches = sum(v[1] for v in prof.values()) // args.steps
+    # dominant kernel = the tcgen05 contraction kernel (its four instantiations together);
+    # it executes 8*N*d*V flops per step because the backward recomputes the logits.
+    exec_tflops = 8.0 * n_live * d * V / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    peak = peaks["sustained"]
+    roofline = {"bound": "tensor", "kernel": "gemm_kernel<lse|grad|dH|dW> (tcgen05, one template)",
+                "achieved": exec_tflops, "peak": peak, "unit": "TFLOP/s",
+                "frac": exec_tflops / peak if exec_tflops else None, "traffic": None,
+                "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
+                "credited_tflops": flops_step / (ms_step * 1e-3) / 1e12,
+                "credited_frac_of_sustained": flops_step / (ms_step * 1e-3) / 1e12 / peaks["sustained"],
+                "credited_frac_of_burst": flops_step / (ms_step * 1e-3) / 1e12 / peaks["burst"],
+                "credited_frac_of_nominal_2250": flops_step / (ms_step * 1e-3) / 1e12 / 2250.0,
+                "contraction_ms_per_step": gemm_ms, "contraction_launches_per_step": gemm_launches,
+                "by_kind_ms_per_step": {k: v[0] / args.steps for k, v in prof.items() if v[1]}}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{wl.name}-scale: d={d}, V={V}, {P} prompts x {wl.samples} rollouts, "
+                                   f"lengths {wl.length}, padded_to={wl.padded_to}, beta={batch['beta_v']}",
+                       "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts",
+                       "l2": "inputs larger than L2 (H, W, g chunk each > 126 MB); no flush needed",
+                       "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "loss": loss_val},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "cpu_baseline": cpu_base}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="7b")
+    ap.add_argument("--beta", type=float, default=1.0)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--ref-rows", type=int, default=256, help="response tokens in the CPU oracle sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

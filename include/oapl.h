@@ -132,6 +132,17 @@ uint64_t oapl_launch_count(void);
 const char* oapl_status_string(int status);
 
 /*
+ * Optional timing of the contraction launches (off by default).  While enabled,
+ * every contraction launch is bracketed by a CUDA event pair on its stream (at most
+ * 2048 launches between reads).  oapl_profile_read waits for those events and sums
+ * the elapsed milliseconds and the launch counts per kind into host arrays of
+ * `kinds` entries: 0 = logits + online log-sum-exp, 1 = logit-gradient chunk,
+ * 2 = dH, 3 = dW, 4 = bring-up GEMM; then clears the record.  Not thread-safe.
+ */
+int oapl_profile_enable(int on);
+int oapl_profile_read(float* ms_by_kind /*host*/, int* launches_by_kind /*host*/, int kinds);
+
+/*
  * Bring-up aid for the tensor-core main loop shared by every contraction above:
  * C[M, N] (f32 row-major, ld = N) = A . B with bf16 operands, through the same
  * TMA/tcgen05 pipeline.  a_mn == 0: A is [M, K] row-major (K contiguous);

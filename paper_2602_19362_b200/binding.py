@@ -20,7 +20,7 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL
 
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
-           "oapl_status_string", "oapl_debug_gemm"]
+           "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -71,6 +71,10 @@ def lib() -> ctypes.CDLL:
         L.oapl_status_string.argtypes = [i32]
         L.oapl_debug_gemm.restype = i32
         L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.oapl_profile_enable.restype = i32
+        L.oapl_profile_enable.argtypes = [i32]
+        L.oapl_profile_read.restype = i32
+        L.oapl_profile_read.argtypes = [vp, vp, i32]
         _lib = L
     return _lib
 
@@ -170,3 +174,22 @@ def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err):
     rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), _ptr(err), _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_debug_gemm")
+
+
+KINDS = ("lse_fwd", "grad_chunk", "dH", "dW", "debug")
+
+
+def oapl_profile_enable(on: bool):
+    rc = lib().oapl_profile_enable(int(on))
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_profile_enable")
+
+
+def oapl_profile_read() -> dict:
+    """{kind: (milliseconds, launches)} since the last read."""
+    ms = (ctypes.c_float * len(KINDS))()
+    cnt = (ctypes.c_int * len(KINDS))()
+    rc = lib().oapl_profile_read(ms, cnt, len(KINDS))
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_profile_read")
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KINDS)}

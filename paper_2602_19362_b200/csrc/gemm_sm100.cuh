@@ -29,9 +29,11 @@ constexpr int kTmemCols = 512;
 constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kErrTimeout = -8;  // OAPL_ERR_DEVICE_TIMEOUT
+constexpr int kFwdTag = 0x0A91;   // written by the loss kernel when a forward has completed
 
 struct GemmParams {
   const int* n_live_ptr;  // device: number of live (compacted) rows; null in debug mode
+  const int* tag_ptr;     // device: forward-completed tag; when set and wrong, no row is live
   int row_begin;          // first compacted row of this call's row range
   int row_cap;            // capacity of the row range (whole problem, or one chunk)
   int R, C;               // sweep schedule: R row blocks x C vocabulary splits per wave
@@ -144,7 +146,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_live = (MODE == MODE_DEBUG) ? 0 : *p.n_live_ptr;
+  int n_live = (MODE == MODE_DEBUG) ? 0 : *p.n_live_ptr;
+  if (MODE != MODE_DEBUG && p.tag_ptr && *p.tag_ptr != kFwdTag) n_live = 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {

@@ -139,6 +139,26 @@ static void pick_sweep(int n_sm, int d, int rb_max, int vtiles, int* R, int* C) 
   *C = c;
 }
 
+// Optional per-contraction timing (off by default): an event pair around every
+// contraction launch, summed per kind by oapl_profile_read.
+constexpr int kProfSlots = 2048;
+static bool g_prof_on = false;
+static int g_prof_used = 0;
+static cudaEvent_t g_prof_ev[kProfSlots][2];
+static int g_prof_kind[kProfSlots];
+static bool g_prof_made = false;
+
+static int prof_begin(int kind, cudaStream_t st) {
+  if (!g_prof_on || g_prof_used >= kProfSlots) return -1;
+  const int s = g_prof_used++;
+  g_prof_kind[s] = kind;
+  cudaEventRecord(g_prof_ev[s][0], st);
+  return s;
+}
+static void prof_end(int slot, cudaStream_t st) {
+  if (slot >= 0) cudaEventRecord(g_prof_ev[slot][1], st);
+}
+
 template <int MODE, int A_MN, int B_MN>
 static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& gp, int grid,
                        cudaStream_t st) {
@@ -150,8 +170,10 @@ static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPar
       return OAPL_ERR_CUDA;
     attr_set = true;
   }
+  const int slot = prof_begin(MODE, st);
   kern<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(a, b, gp);
   OAPL_LAUNCHED();
+  prof_end(slot, st);
   return cudaGetLastError() == cudaSuccess ? OAPL_OK : OAPL_ERR_CUDA;
 }
 
@@ -364,7 +386,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(w + c.Hc);
   __nv_bfloat16* G = reinterpret_cast<__nv_bfloat16*>(w + c.G);
 
-  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH));
+  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH), state);
   CKL();
   if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
 
@@ -381,6 +403,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   GemmParams gp;
   memset(&gp, 0, sizeof(gp));
   gp.n_live_ptr = &state->n_live;
+  gp.tag_ptr = &state->fwd_tag;
   gp.row_cap = c.chunk_rows;
   gp.d = p->d;
   gp.V = p->V;
@@ -409,6 +432,31 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
     rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, gp, n_sm, st);
     if (rc != OAPL_OK) return rc;
   }
+  return OAPL_OK;
+}
+
+int oapl_profile_enable(int on) {
+  if (on && !g_prof_made) {
+    for (int i = 0; i < kProfSlots; ++i)
+      for (int j = 0; j < 2; ++j)
+        if (cudaEventCreate(&g_prof_ev[i][j]) != cudaSuccess) return OAPL_ERR_CUDA;
+    g_prof_made = true;
+  }
+  g_prof_on = on != 0;
+  g_prof_used = 0;
+  return OAPL_OK;
+}
+
+int oapl_profile_read(float* ms_by_kind, int* launches_by_kind, int kinds) {
+  if (!ms_by_kind || !launches_by_kind || kinds <= 0) return OAPL_ERR_INVALID_ARG;
+  for (int k = 0; k < kinds; ++k) { ms_by_kind[k] = 0.f; launches_by_kind[k] = 0; }
+  for (int s = 0; s < g_prof_used; ++s) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(g_prof_ev[s][1]) != cudaSuccess) return OAPL_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms, g_prof_ev[s][0], g_prof_ev[s][1]) != cudaSuccess) return OAPL_ERR_CUDA;
+    if (g_prof_kind[s] < kinds) { ms_by_kind[g_prof_kind[s]] += ms; launches_by_kind[g_prof_kind[s]] += 1; }
+  }
+  g_prof_used = 0;
   return OAPL_OK;
 }
 

@@ -143,7 +143,8 @@ __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ H, const in
 
 // ---- zero the dH rows of masked positions -------------------------------------------
 __global__ void zero_dead_rows_kernel(const uint8_t* __restrict__ mask, long long N, int d,
-                                      __nv_bfloat16* __restrict__ dH) {
+                                      __nv_bfloat16* __restrict__ dH, DevState* st) {
+  if (blockIdx.x == 0 && threadIdx.x == 0 && st->fwd_tag != 0x0A91) set_error(&st->status, -10);
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int vec = d >> 3;
@@ -282,7 +283,7 @@ __global__ void loss_kernel(const float* __restrict__ reward, const int* __restr
     double t = 0.0;
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
     *loss = (float)((double)loss_scale * t);
-    st->fwd_tag = 0x0A91;
+    st->fwd_tag = 0x0A91;  // = kFwdTag of the contraction kernel
   }
 }
 
