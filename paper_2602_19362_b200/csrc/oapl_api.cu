@@ -233,7 +233,7 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   scan_blocks_kernel<<<1, 1024, 0, st>>>(block_cnt, c.nblk, block_off, state);
   CKL();
   write_live_kernel<<<c.nblk, kScanBlock, 0, st>>>(p->mask, p->seq_id, p->targets,
-                                                   with_q ? p->logp_inf : nullptr, p->N, block_off,
+                                                   with_q ? p->logp_inf : nullptr, p->N, p->S, block_off,
                                                    live_rows, tgt_c, seq_c, q_c);
   CKL();
   seq_bounds_kernel<<<n_sm * 2, 256, 0, st>>>(seq_c, state, cstart, cend);

@@ -80,7 +80,7 @@ __global__ void scan_blocks_kernel(const int* __restrict__ block_cnt, int nblk,
 // ---- pass 3: write the compacted per-row arrays --------------------------------
 __global__ void write_live_kernel(const uint8_t* __restrict__ mask, const int* __restrict__ seq_id,
                                   const int* __restrict__ targets, const float* __restrict__ logp_inf,
-                                  long long N, const int* __restrict__ block_off,
+                                  long long N, int S, const int* __restrict__ block_off,
                                   int* __restrict__ live_rows, int* __restrict__ tgt_c,
                                   int* __restrict__ seq_c, float* __restrict__ q_c) {
   __shared__ int warp_sum[32];
@@ -105,7 +105,9 @@ __global__ void write_live_kernel(const uint8_t* __restrict__ mask, const int* _
     const int i = block_off[blockIdx.x] + (warp ? warp_sum[warp - 1] : 0) + in_warp;
     live_rows[i] = (int)n;
     tgt_c[i] = targets[n];
-    seq_c[i] = seq_id[n];
+    // an out-of-range id has already raised the error word; clamp so that no later
+    // kernel indexes outside its per-sequence arrays
+    seq_c[i] = min(max(seq_id[n], 0), S - 1);
     q_c[i] = logp_inf ? logp_inf[n] : 0.f;
   }
 }

@@ -1,0 +1,72 @@
+"""The 7B-scale configuration at full size, in the launch configuration the benchmark
+times.  The whole problem is out of reach for a CPU (about 1e15 flops), so the oracle
+checks sampled outputs it can compute one by one, and properties that hold at any size
+cover the rest."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oapl_oracle as orc
+from paper_2602_19362_b200 import synth
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def test_7b_full_size_sampled_rows_and_invariants():
+    wl = synth.WORKLOADS["7b"]
+    dev = synth.make_batch(wl, seed=0, device="cuda", beta=1.0)
+    out = hp.run_gpu(dev)
+    assert out["status"] == 0 and out["n_live"] == dev["live_tokens"]
+    N, S, P, d, V = (dev[k] for k in ("N", "S", "P", "d", "V"))
+    mask = dev["mask"].bool()
+
+    # --- sampled live rows (first, last, tile and chunk boundaries, random): token log-prob and dH row
+    live = torch.nonzero(mask).flatten()
+    g = torch.Generator().manual_seed(0)
+    pick = torch.cat([torch.tensor([0, 1, 127, 128, 9471, 9472, live.numel() - 1]),
+                      torch.randint(0, live.numel(), (41,), generator=g)])
+    rows = live[pick.to(live.device)]
+    Wd = orc.bf16_bits_to_f64(synth.bf16_bits(dev["W"]))
+    Hs = orc.bf16_bits_to_f64(synth.bf16_bits(dev["H"][rows]))
+    tg = hp.npy(dev["targets"][rows])
+    lp_ref, _ = orc.token_logprobs(Hs, Wd, tg, np.ones(len(rows), dtype=np.uint8))
+    assert np.abs(hp.npy(out["token_logp"][rows]) - lp_ref).max() <= hp.TOL_TOKEN
+
+    # --- O(N) stages re-run by the oracle on the library's own token log-probs: exact check of
+    #     the segmented sums, Eq. 2 and Eq. 3 at full size
+    tok = hp.npy(out["token_logp"]).astype(np.float64)
+    s, D, T = orc.sequence_sums(tok, hp.npy(dev["logp_inf"]), hp.npy(dev["mask"]), hp.npy(dev["seq_id"]), S)
+    tail = orc.loss_from_sums(D, hp.npy(dev["reward"]), hp.npy(dev["group_id"]), P, 1.0, 1.0, dev["loss_scale"])
+    assert np.allclose(hp.npy(out["seq_logp"]), s, rtol=1e-6)
+    assert np.allclose(hp.npy(out["vhat"]), tail["vhat"], rtol=1e-6, atol=1e-7)
+    assert np.allclose(hp.npy(out["delta"]), tail["delta"], rtol=1e-4, atol=1e-4)
+    assert float(out["loss"]) == pytest.approx(tail["loss"], rel=1e-5)
+
+    # --- dH of the sampled rows from the oracle's own coefficients of those rows' sequences
+    coef = tail["coef"]
+    sid = hp.npy(dev["seq_id"][rows])
+    dH_ref, _ = orc.loss_bwd(Hs, Wd, tg, np.ones(len(rows), dtype=np.uint8), np.arange(len(rows)), coef[sid])
+    got = hp.npy(out["dH"][rows].float()).astype(np.float64)
+    assert hp.fro_rel(got, dH_ref) <= hp.TOL_FRO
+    for i in range(len(rows)):
+        assert hp.fro_rel(got[i], dH_ref[i]) <= 2 * hp.TOL_FRO
+
+    # --- properties that hold at any size
+    dH, dW = out["dH"], out["dW"]
+    assert torch.isfinite(dW).all() and torch.isfinite(dH.float()).all()
+    assert float(dH[~mask].float().abs().max()) == 0.0                       # masked rows exactly zero
+    col = dW.double().sum(dim=0)                                             # softmax rows sum to 1
+    assert float(col.abs().max()) <= 1e-3 * float(dW.double().abs().sum(dim=0).max())
+    # <dH, H> = <dW, W> = sum_nv g[n,v] z[n,v].  Both sides use the same bf16 g, so what
+    # separates them is the bf16 rounding of the dH output: independent relative errors of
+    # at most 2^-9 per element, i.e. a standard deviation of about 2^-9/sqrt(3) * ||dH o H||_2
+    # on the sum; allow six of those.
+    lhs, sq = 0.0, 0.0
+    for r0 in range(0, N, 65536):
+        prod = dH[r0:r0 + 65536].double() * dev["H"][r0:r0 + 65536].double()
+        lhs += float(prod.sum())
+        sq += float((prod * prod).sum())
+    rhs = float((dW.double() * dev["W"].double()).sum())
+    sigma = 2.0 ** -9 / np.sqrt(3.0) * np.sqrt(sq)
+    assert abs(lhs - rhs) <= 6.0 * sigma + 1e-4 * abs(rhs), (lhs, rhs, sigma)

@@ -48,3 +48,12 @@ def test_value_estimate_entry_point():
         want = orc.value_estimate(reward.numpy(), group_id.numpy(), P, beta)
         assert np.allclose(vhat.cpu().numpy(), want, rtol=2e-6, atol=2e-6)
         assert vhat[P - 1].item() == 0.0
+
+
+def test_many_chunks_and_waves_in_the_default_launch_configuration():
+    # about 20k response tokens: three default row chunks, several waves of row blocks
+    # per chunk, sequences straddling tiles and chunks; small d and V keep the oracle fast
+    wl = dataclasses.replace(synth.WORKLOADS["tiny"], prompts=16, samples=8, length=("uniform", 64, 256),
+                             padded_to=256, d=256, V=4096 + 72)
+    cpu, out, ref = _check(wl, seed=11)
+    assert cpu["live_tokens"] > 2 * 9472
