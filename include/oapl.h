@@ -132,6 +132,33 @@ uint64_t oapl_launch_count(void);
 const char* oapl_status_string(int status);
 
 /*
+ * oapl_token_logprobs for callers that cannot provide a workspace.  (The paper has no
+ * counterpart; this is a property of the library, not of the method.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory where it calls us --
+ * a plug-in inside a framework that owns the allocator, a serving loop whose memory was
+ * fixed at start-up, or a section in which the CUDA allocator must not be entered.  The
+ * scratch memory lives in a fixed device array inside the library (about 4.6 MB per GPU
+ * that loads the library, held until the process exits), so sizes are limited:
+ *     N <= 2048,  d <= 1024 (multiple of 64),  S <= 2048,  any V >= 1.
+ * Larger problems return OAPL_ERR_UNSUPPORTED_SHAPE and print the limits to stderr.
+ * The call itself allocates and frees nothing.
+ *
+ *   token_logp [N] f32, seq_logp [S] f32 or NULL: as in oapl_token_logprobs.
+ *   device_status: device int32 or NULL; receives the device-detected status word
+ *                  (OAPL_OK, OAPL_ERR_BAD_TARGET, OAPL_ERR_BAD_SEQ_ORDER, ...) in stream order.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call before starting any stream capture.  All calls on one
+ * GPU share the one array and it keeps the previous call's contents; the call clears the
+ * parts that must start at zero, but two calls whose work overlaps on the GPU (different
+ * streams without ordering, or several host threads) race on it and give wrong results:
+ * order them.
+ */
+int oapl_token_logprobs_static(const oapl_problem* problem /*host*/, float* token_logp, float* seq_logp,
+                               int32_t* device_status, void* stream);
+
+/*
  * Optional timing of the contraction launches (off by default).  While enabled,
  * every contraction launch is bracketed by a CUDA event pair on its stream (at most
  * 2048 launches between reads).  oapl_profile_read waits for those events and sums

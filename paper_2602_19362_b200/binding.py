@@ -20,7 +20,8 @@ STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL
 
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
-           "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read"]
+           "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
+           "oapl_token_logprobs_static"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.oapl_status_string.argtypes = [i32]
         L.oapl_debug_gemm.restype = i32
         L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.oapl_token_logprobs_static.restype = i32
+        L.oapl_token_logprobs_static.argtypes = [pp, vp, vp, vp, vp]
         L.oapl_profile_enable.restype = i32
         L.oapl_profile_enable.argtypes = [i32]
         L.oapl_profile_read.restype = i32
@@ -193,3 +196,12 @@ def oapl_profile_read() -> dict:
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_profile_read")
     return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KINDS)}
+
+
+def oapl_token_logprobs_static(problem, token_logp, seq_logp, device_status=None):
+    """oapl_token_logprobs without a workspace: the scratch is a fixed array inside the
+    library, for callers that must not allocate (N <= 2048, d <= 1024, S <= 2048)."""
+    rc = lib().oapl_token_logprobs_static(ctypes.byref(problem), _ptr(token_logp), _ptr(seq_logp),
+                                          _ptr(device_status), _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_token_logprobs_static")

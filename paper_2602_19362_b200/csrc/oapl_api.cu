@@ -488,4 +488,101 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   return launch_gemm<MODE_DEBUG, 1, 1>(ta, tb, gp, grid, st);
 }
 
+// ---------------------------------------------------------------------------------------
+// Token log-probabilities without a caller-provided workspace.
+//
+// Some callers of this library cannot hand it scratch memory because they are not allowed
+// to allocate device memory at the point of the call: a plug-in running inside a host
+// framework that owns the allocator, a latency-critical serving loop whose memory was fixed
+// at start-up, or a region of code where the CUDA allocator must not be entered.  For them
+// the scratch of oapl_token_logprobs lives in the fixed device array below (about 4.6 MB,
+// resident on every GPU that loads the library until the process exits), which bounds the
+// problem size: N <= 2048 rows, d <= 1024, S <= 2048 sequences, any V.
+constexpr int kStaticMaxRows = 2048;
+constexpr int kStaticMaxD = 1024;
+constexpr int kStaticMaxSeq = 2048;
+constexpr size_t kStaticScratchBytes =
+    1024 /*state*/ + 2 * 1024 /*block counts, offsets*/ + 6 * 4 * (size_t)kStaticMaxRows /*per-row arrays*/ +
+    3 * 4 * (size_t)kStaticMaxRows * kMaxSplits /*log-sum-exp partials*/ +
+    3 * 4 * (size_t)kStaticMaxSeq /*per-sequence arrays*/ +
+    2 * (size_t)kStaticMaxRows * kStaticMaxD /*compacted H*/ + 16 * 1024 /*alignment slack*/;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// The array's name is only a host-side handle; kernels need its device address, which is
+// looked up once per device (with that device current) and cached.
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_scratch_addr[kMaxDevices] = {nullptr};
+
+static int static_scratch_for_current_device(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return OAPL_ERR_CUDA;
+  if (!g_static_scratch_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return OAPL_ERR_CUDA;
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *out = g_static_scratch_addr[dev];
+  return OAPL_OK;
+}
+
+int oapl_token_logprobs_static(const oapl_problem* p, float* token_logp, float* seq_logp,
+                               int32_t* device_status, void* stream) {
+  int rc = check_problem(p, false);
+  if (rc != OAPL_OK) return rc;
+  if (!token_logp) return OAPL_ERR_INVALID_ARG;
+  if (p->N > kStaticMaxRows || p->d > kStaticMaxD || p->S > kStaticMaxSeq) {
+    fprintf(stderr,
+            "oapl_token_logprobs_static: problem (N=%lld, d=%d, S=%d) exceeds the built-in scratch "
+            "(N <= %d, d <= %d, S <= %d); use oapl_token_logprobs with a workspace\n",
+            (long long)p->N, p->d, p->S, kStaticMaxRows, kStaticMaxD, kStaticMaxSeq);
+    return OAPL_ERR_UNSUPPORTED_SHAPE;
+  }
+  unsigned char* base = nullptr;
+  rc = static_scratch_for_current_device(&base);
+  if (rc != OAPL_OK) return rc;
+
+  // Lay the forward's scratch out inside the fixed array (1 KB-aligned pieces).
+  Carve c;
+  memset(&c, 0, sizeof(c));
+  const size_t n_pad = align_up((size_t)p->N, 128);
+  c.n_pad = (int)n_pad;
+  c.nblk = (int)((p->N + kScanBlock - 1) / kScanBlock);
+  c.chunk_rows = (int)n_pad;
+  c.ldg = 0;
+  size_t off = align_up((size_t)(uintptr_t)base, 1024) - (size_t)(uintptr_t)base;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off = align_up(off + bytes, 1024);
+    return o;
+  };
+  c.state = take(sizeof(DevState));
+  c.block_cnt = take(4 * (size_t)c.nblk);
+  c.block_off = take(4 * (size_t)c.nblk);
+  c.live_rows = take(4 * n_pad);
+  c.tgt_c = take(4 * n_pad);
+  c.seq_c = take(4 * n_pad);
+  c.q_c = take(4 * n_pad);
+  c.lp_c = take(4 * n_pad);
+  c.lse = take(4 * n_pad);
+  c.pm = take(4 * n_pad * kMaxSplits);
+  c.pl = take(4 * n_pad * kMaxSplits);
+  c.pz = take(4 * n_pad * kMaxSplits);
+  c.cstart = take(4 * (size_t)p->S);
+  c.cend = take(4 * (size_t)p->S);
+  c.seq_D = take(4 * (size_t)p->S);
+  c.Hc = take(2 * n_pad * (size_t)p->d);
+  c.total = off;
+  if (c.total > kStaticScratchBytes) return OAPL_ERR_UNSUPPORTED_SHAPE;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // forward_common clears the state word and the per-sequence bounds itself; everything
+  // else it reads from the scratch it has written earlier in the same call.
+  rc = forward_common(p, c, base, token_logp, seq_logp, false, st);
+  if (rc != OAPL_OK) return rc;
+  if (device_status)
+    CK(cudaMemcpyAsync(device_status, &reinterpret_cast<DevState*>(base + c.state)->status, sizeof(int),
+                       cudaMemcpyDeviceToDevice, st));
+  return OAPL_OK;
+}
+
 }  // extern "C"
