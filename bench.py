@@ -196,6 +196,10 @@ def run_cuda(args) -> None:
                     "sample": desc, "seconds": dt}
 
     wl = synth.WORKLOADS[args.workload]
+    if args.prompts or args.samples:      # reduced copies of the workload, for profiler captures
+        import dataclasses
+        wl = dataclasses.replace(wl, prompts=args.prompts or wl.prompts, samples=args.samples or wl.samples,
+                                 name=wl.name + "-reduced")
     # data-parallel over prompts: every rank holds its own groups (weak scaling), W replicated
     batch = synth.make_batch(wl, seed=args.seed + rank, device=str(dev), beta=args.beta)
     N, S, P, d, V = (batch[k] for k in ("N", "S", "P", "d", "V"))
@@ -337,6 +341,8 @@ def main() -> None:
     ap.add_argument("--beta", type=float, default=1.0)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--ref-rows", type=int, default=256, help="response tokens in the CPU oracle sample")
+    ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (profiling)")
+    ap.add_argument("--samples", type=int, default=0, help="override rollouts per prompt (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
