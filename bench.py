@@ -205,7 +205,8 @@ def run_cuda(args) -> None:
     N, S, P, d, V = (batch[k] for k in ("N", "S", "P", "d", "V"))
     n_live = batch["live_tokens"]
     prob = B.make_problem(batch)
-    ws = B.alloc_workspace(prob, device=dev)
+    fused = args.path == "single-call"
+    ws = B.alloc_workspace(prob, B.OAPL_FLAG_FUSED if fused else 0, device=dev)
     loss = torch.zeros(1, device=dev)
     seq_logp = torch.zeros(S, device=dev)
     vhat = torch.zeros(P, device=dev)
@@ -214,8 +215,11 @@ def run_cuda(args) -> None:
     dW = torch.empty(V, d, dtype=torch.float32, device=dev)
 
     def step():
-        B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
-        B.oapl_loss_bwd(prob, dH, dW, False, ws)
+        if fused:
+            B.oapl_loss_fwd_bwd(prob, loss, seq_logp, vhat, delta, None, dH, dW, False, ws)
+        else:
+            B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
+            B.oapl_loss_bwd(prob, dH, dW, False, ws)
 
     def barrier():
         if world > 1:
@@ -236,19 +240,16 @@ def run_cuda(args) -> None:
         sampler.start()
     B.oapl_profile_enable(True)
     launches0 = B.oapl_launch_count()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
     ev[0].record()
     for k in range(args.steps):
-        B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
-        ev[2 * k + 1].record()
-        B.oapl_loss_bwd(prob, dH, dW, False, ws)
-        ev[2 * k + 2].record()
+        step()
+        ev[k + 1].record()
     barrier()
     launches = B.oapl_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[2 * args.steps])
-    fwd_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
-    bwd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
     prof = B.oapl_profile_read()
     B.oapl_profile_enable(False)
     clocks = sampler.stop() if rank == 0 else None
@@ -302,11 +303,14 @@ def run_cuda(args) -> None:
     flops_step = 6.0 * n_live * d * V          # credited: logits, dH, dW
     gemm_ms = sum(v[0] for v in prof.values()) / args.steps
     gemm_launches = sum(v[1] for v in prof.values()) // args.steps
-    # dominant kernel = the tcgen05 contraction kernel (its four instantiations together);
-    # it executes 8*N*d*V flops per step because the backward recomputes the logits.
-    exec_tflops = 8.0 * n_live * d * V / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+    # dominant kernel = the tcgen05 contraction kernel (all its instantiations together).  The
+    # single-call path executes 6*N*d*V flops per step; the two-call path recomputes the logits
+    # in the backward and executes 8*N*d*V.
+    exec_factor = 6.0 if fused else 8.0
+    exec_tflops = exec_factor * n_live * d * V / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     peak = peaks["sustained"]
-    roofline = {"bound": "tensor", "kernel": "gemm_kernel<lse|grad|dH|dW> (tcgen05, one template)",
+    roofline = {"bound": "tensor", "kernel": "gemm_kernel (tcgen05, one template: " + ("lse_e|dW|dH)" if fused else "lse|grad|dH|dW)"),
+                "executed_flops_per_step": exec_factor * n_live * d * V,
                 "achieved": exec_tflops, "peak": peak, "unit": "TFLOP/s",
                 "frac": exec_tflops / peak if exec_tflops else None, "traffic": None,
                 "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
@@ -323,7 +327,8 @@ def run_cuda(args) -> None:
                                    f"lengths {wl.length}, padded_to={wl.padded_to}, beta={batch['beta_v']}",
                        "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts",
                        "l2": "inputs larger than L2 (H, W, g chunk each > 126 MB); no flush needed",
-                       "fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "loss": loss_val},
+                       "api": "oapl_loss_fwd_bwd" if fused else "oapl_loss_fwd + oapl_loss_bwd",
+                       "step_ms": step_ms, "loss": loss_val},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu_base}
     print(json.dumps(line), flush=True)
@@ -343,6 +348,8 @@ def main() -> None:
     ap.add_argument("--ref-rows", type=int, default=256, help="response tokens in the CPU oracle sample")
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (profiling)")
     ap.add_argument("--samples", type=int, default=0, help="override rollouts per prompt (profiling)")
+    ap.add_argument("--path", default="single-call", choices=["single-call", "two-calls"],
+                    help="oapl_loss_fwd_bwd (no recompute) or oapl_loss_fwd + oapl_loss_bwd")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

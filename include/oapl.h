@@ -40,11 +40,13 @@ typedef enum {
   OAPL_ERR_NONFINITE_INPUT = -7,     /* device: non-finite reward, or group_id outside [0,P) */
   OAPL_ERR_DEVICE_TIMEOUT = -8,      /* device: a bounded pipeline wait expired */
   OAPL_ERR_CUDA = -9,                /* a CUDA runtime/driver call failed */
-  OAPL_ERR_BAD_STATE = -10           /* oapl_loss_bwd without a matching oapl_loss_fwd in ws */
+  OAPL_ERR_BAD_STATE = -10,          /* oapl_loss_bwd without a matching oapl_loss_fwd in ws */
+  OAPL_ERR_SEQUENCE_TOO_LONG = -11   /* device: oapl_loss_fwd_bwd met a sequence longer than its staging capacity */
 } oapl_status;
 
 /* flags */
 #define OAPL_FLAG_NONE 0
+#define OAPL_FLAG_FUSED 1 /* oapl_workspace_bytes: size the workspace for oapl_loss_fwd_bwd */
 
 /*
  * One batch, as the paper states the problem (Eq. 2 / Eq. 3): for every prompt x a
@@ -118,6 +120,27 @@ int oapl_loss_fwd(const oapl_problem* problem /*host*/, float* loss, float* seq_
 int oapl_loss_bwd(const oapl_problem* problem /*host*/, void* dH, float* dW, int accumulate_dW,
                   void* ws, size_t ws_bytes, int flags, void* stream);
 
+/*
+ * Eq. 3 forward and gradient in one call, without recomputing the logits in the backward.
+ * Same inputs and outputs as oapl_loss_fwd followed by oapl_loss_bwd (same definitions:
+ * Eq. 2, Eq. 3 and g = c_i * mask * (onehot - softmax)), but the work is organised by ranges
+ * of whole sequences: for each range the logits pass stores e = exp(z - zref_row) as bf16
+ * (zref_row = target logit + 40), the per-sequence coefficients of the range follow from
+ * its log-probabilities, and since g = -c_i * e' / sum_v e (e' = e with the target entry
+ * lowered by sum_v e) both gradient contractions read the staged e' directly:
+ * dH = rowscale(e'.W), dW += e'^T.(scaled H).  Executed work is 6*N*d*V flops instead of 8.
+ *
+ * Workspace: oapl_workspace_bytes(problem, OAPL_FLAG_FUSED).  It holds e for 32768 rows
+ * (2 bytes * round_up(V,256) each; OAPL_STAGE_ROWS in the environment changes the count), so
+ * it does not grow with N*V; a sequence with more live rows than that cannot be staged and
+ * raises OAPL_ERR_SEQUENCE_TOO_LONG in the status word (outputs are then not meaningful;
+ * use the two separate calls).  A target whose probability under the policy is below
+ * e^-128 is outside the range of the staged exponentials.
+ */
+int oapl_loss_fwd_bwd(const oapl_problem* problem /*host*/, float* loss, float* seq_logp, float* vhat,
+                      float* delta /*may be NULL*/, float* token_logp /*may be NULL*/, void* dH, float* dW,
+                      int accumulate_dW, void* ws, size_t ws_bytes, int flags, void* stream);
+
 /* Synchronises `stream` and returns the status word the device recorded in `ws`
  * since the last forward call (OAPL_OK if none). */
 int oapl_get_last_status(void* ws, void* stream);
@@ -164,7 +187,7 @@ int oapl_token_logprobs_static(const oapl_problem* problem /*host*/, float* toke
  * 2048 launches between reads).  oapl_profile_read waits for those events and sums
  * the elapsed milliseconds and the launch counts per kind into host arrays of
  * `kinds` entries: 0 = logits + online log-sum-exp, 1 = logit-gradient chunk,
- * 2 = dH, 3 = dW, 4 = bring-up GEMM; then clears the record.  Not thread-safe.
+ * 2 = dH, 3 = dW, 4 = bring-up GEMM, 5 = logits + staged exponentials; then clears the record.  Not thread-safe.
  */
 int oapl_profile_enable(int on);
 int oapl_profile_read(float* ms_by_kind /*host*/, int* launches_by_kind /*host*/, int kinds);

@@ -16,12 +16,13 @@ LIB_PATH = os.path.join(_HERE, "liboapl.so")
 OAPL_OK = 0
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL",
           -4: "UNSUPPORTED_SHAPE", -5: "BAD_TARGET", -6: "BAD_SEQ_ORDER", -7: "NONFINITE_INPUT",
-          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE"}
+          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE", -11: "SEQUENCE_TOO_LONG"}
+OAPL_FLAG_FUSED = 1
 
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
-           "oapl_token_logprobs_static"]
+           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -72,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.oapl_status_string.argtypes = [i32]
         L.oapl_debug_gemm.restype = i32
         L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.oapl_loss_fwd_bwd.restype = i32
+        L.oapl_loss_fwd_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_token_logprobs_static.restype = i32
         L.oapl_token_logprobs_static.argtypes = [pp, vp, vp, vp, vp]
         L.oapl_profile_enable.restype = i32
@@ -179,7 +182,7 @@ def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err):
         raise OaplError(rc, "oapl_debug_gemm")
 
 
-KINDS = ("lse_fwd", "grad_chunk", "dH", "dW", "debug")
+KINDS = ("lse_fwd", "grad_chunk", "dH", "dW", "debug", "lse_e")
 
 
 def oapl_profile_enable(on: bool):
@@ -205,3 +208,11 @@ def oapl_token_logprobs_static(problem, token_logp, seq_logp, device_status=None
                                           _ptr(device_status), _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_token_logprobs_static")
+
+
+def oapl_loss_fwd_bwd(problem, loss, seq_logp, vhat, delta, token_logp, dH, dW, accumulate_dW, ws, flags=0):
+    rc = lib().oapl_loss_fwd_bwd(ctypes.byref(problem), _ptr(loss), _ptr(seq_logp), _ptr(vhat), _ptr(delta),
+                                 _ptr(token_logp), _ptr(dH), _ptr(dW), int(accumulate_dW), _ptr(ws),
+                                 ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_loss_fwd_bwd")

@@ -1,45 +1,53 @@
 // One persistent, warp-specialised tcgen05 contraction kernel, instantiated with
-// five epilogues:
-//   MODE_LSE   z = H.W^T tile by tile; per-row running (max, sum-exp) and target logit
-//   MODE_GRAD  z recomputed; g = c*(onehot - softmax) written as a bf16 row chunk
-//   MODE_DH    dH = g . W      (contraction over the vocabulary)
-//   MODE_DW    dW (+)= g^T . H (contraction over the rows of the chunk)
-//   MODE_DEBUG plain C = A.B for bring-up of the four operand-major combinations
+// six epilogues:
+//   MODE_LSE    z = H.W^T tile by tile; per-row running (max, sum-exp) and target logit
+//   MODE_GRAD   z recomputed; g = c*(onehot - softmax) written as a bf16 row chunk
+//   MODE_DH     dH = g . W      (contraction over the vocabulary), optional per-row scale
+//   MODE_DW     dW (+)= g^T . H (contraction over the rows of the range)
+//   MODE_LSE_E  z tile by tile; e = exp(z - zref_row) staged as bf16 for a range of whole
+//               sequences, per-row sum of e and target logit (no recompute in the backward)
+//   MODE_DEBUG  plain C = A.B for bring-up of the four operand-major combinations
 //
 // CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM and issues the UMMAs,
 // warps 2..5 are the epilogue (one TMEM lane quadrant each).  Tile 128 x 256 x 64,
 // four shared-memory stages, two 256-column fp32 accumulators in TMEM so that the
-// epilogue of tile j overlaps the main loop of tile j+1.
+// epilogue of tile j overlaps the main loop of tile j+1.  bf16 tiles leave through
+// shared memory and TMA stores.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "sm100_ptx.cuh"
+#include "sweep_schedule.cuh"
 
 namespace oapl {
 
-enum { MODE_LSE = 0, MODE_GRAD = 1, MODE_DH = 2, MODE_DW = 3, MODE_DEBUG = 4 };
+enum { MODE_LSE = 0, MODE_GRAD = 1, MODE_DH = 2, MODE_DW = 3, MODE_DEBUG = 4, MODE_LSE_E = 5 };
 
 constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
 constexpr int kABytes = kBM * kBK * 2;  // 16 KB
 constexpr int kBBytes = kBN * kBK * 2;  // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kOutBytes = kBM * 64 * 2;  // one 128 x 64 bf16 output piece (16 KB), two of them
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kGemmSmemBytes = size_t(kStages) * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr size_t kGemmSmemBytes =
+    size_t(kStages) * kStageBytes + 2 * kOutBytes + 1024 /*align*/ + 256 /*barriers*/;
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kErrTimeout = -8;  // OAPL_ERR_DEVICE_TIMEOUT
-constexpr int kFwdTag = 0x0A91;   // written by the loss kernel when a forward has completed
+constexpr int kFwdTag = 0x0A91;  // written by the loss kernel when a forward has completed
 
 struct GemmParams {
   const int* n_live_ptr;  // device: number of live (compacted) rows; null in debug mode
   const int* tag_ptr;     // device: forward-completed tag; when set and wrong, no row is live
+  const int* range_ptr;   // device: {row_begin, row_end} of this launch; null = use the two below
   int row_begin;          // first compacted row of this call's row range
   int row_cap;            // capacity of the row range (whole problem, or one chunk)
   int R, C;               // sweep schedule: R row blocks x C vocabulary splits per wave
   int d, V;
-  int ldg;                // leading dimension of the g chunk (elements)
-  // MODE_LSE outputs: per (row, split) partials
+  int ldg;                // leading dimension of the staged bf16 chunk (elements)
+  // sweep outputs: per (row, split) partials, kMaxSplits slots per row
   float* pm;
   float* pl;
   float* pz;
@@ -47,8 +55,9 @@ struct GemmParams {
   const int* tgt_c;
   const int* seq_c;
   const float* lse;
-  const float* coef;  // per sequence
-  __nv_bfloat16* G;   // chunk [row_cap, ldg]
+  const float* zref;      // MODE_LSE_E: per-row reference subtracted before the exponential
+  const float* rowscale;  // MODE_DH: optional per-row factor applied to the output
+  const float* coef;      // per sequence
   const int* live_rows;
   __nv_bfloat16* dH;  // [N, d]
   float* dW;          // [V, d]
@@ -66,53 +75,68 @@ struct Tile {
   int first, last, split;
 };
 
+// Tile j of this CTA for rows [row_begin, row_end) of the compacted row space.
 template <int MODE>
-__device__ __forceinline__ bool get_tile(const GemmParams& p, int n_live, int j, Tile& t) {
+__device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int row_end, int j,
+                                         Tile& t) {
   t.first = t.last = 1;
   t.split = 0;
-  if (MODE == MODE_LSE || MODE == MODE_GRAD) {
+  const int rows = row_end - row_begin;
+  if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
+    if (rows <= 0) return false;
     const int VT = (p.V + kBN - 1) / kBN;
+    const int nrb = (rows + kBM - 1) / kBM;
+    const SweepShape sh = sweep_shape(nrb, p.R, p.C, VT);
+    // complete waves: this CTA is (row block rbi, split s) of every wave
     const int rbi = blockIdx.x % p.R, s = blockIdx.x / p.R;
-    if (s >= p.C) return false;
-    const int vt0 = (int)((long long)VT * s / p.C), vt1 = (int)((long long)VT * (s + 1) / p.C);
-    const int per = vt1 - vt0;
-    if (per <= 0) return false;
-    const int wave = j / per, off = j - wave * per;
-    int row_end = p.row_begin + p.row_cap;
-    if (row_end > n_live) row_end = n_live;
-    const int rb = p.row_begin / kBM + wave * p.R + rbi;
-    if (rb * kBM >= row_end) return false;
-    t.m0 = rb * kBM;
+    int vt0 = (int)((long long)VT * s / p.C), vt1 = (int)((long long)VT * (s + 1) / p.C);
+    int per = (s < p.C) ? vt1 - vt0 : 0;
+    const int main_tiles = sh.nfull * per;
+    int rbk, off;
+    if (j < main_tiles) {
+      const int wave = j / per;
+      off = j - wave * per;
+      rbk = wave * p.R + rbi;
+      t.split = s;
+    } else {
+      // tail wave: rem row blocks x Ct splits
+      if (sh.rem == 0) return false;
+      const int rbt = blockIdx.x % sh.rem, st = blockIdx.x / sh.rem;
+      if (st >= sh.Ct) return false;
+      vt0 = (int)((long long)VT * st / sh.Ct);
+      vt1 = (int)((long long)VT * (st + 1) / sh.Ct);
+      per = vt1 - vt0;
+      off = j - main_tiles;
+      if (off >= per) return false;
+      rbk = sh.nfull * p.R + rbt;
+      t.split = st;
+    }
+    t.m0 = row_begin + rbk * kBM;
     t.n0 = (vt0 + off) * kBN;
     t.ka0 = t.kb0 = 0;
     t.nk = p.d / kBK;
     t.first = (off == 0);
     t.last = (off == per - 1);
-    t.split = s;
     return true;
   } else if (MODE == MODE_DH) {
-    int rows = n_live - p.row_begin;
-    if (rows > p.row_cap) rows = p.row_cap;
     if (rows <= 0) return false;
     const int MB = (rows + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
     const int tix = blockIdx.x + j * gridDim.x;
     if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kBM;  // row inside the chunk
+    t.m0 = (tix / NB) * kBM;  // row inside the staged chunk
     t.n0 = (tix % NB) * kBN;
     t.ka0 = t.kb0 = 0;
     t.nk = (p.V + kBK - 1) / kBK;
     return true;
   } else if (MODE == MODE_DW) {
-    int rows = n_live - p.row_begin;
-    if (rows > p.row_cap) rows = p.row_cap;
     if (rows <= 0) return false;
     const int MB = (p.V + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
     const int tix = blockIdx.x + j * gridDim.x;
     if (tix >= MB * NB) return false;
     t.m0 = (tix / NB) * kBM;  // vocabulary row
     t.n0 = (tix % NB) * kBN;
-    t.ka0 = 0;            // g chunk rows are chunk-relative
-    t.kb0 = p.row_begin;  // compacted H rows are absolute
+    t.ka0 = 0;          // staged chunk rows are range-relative
+    t.kb0 = row_begin;  // compacted H rows are absolute
     t.nk = (rows + kBK - 1) / kBK;
     return true;
   } else {
@@ -127,16 +151,42 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int n_live, int j,
   }
 }
 
+// Write one thread's 64 bf16 values (32 packed words) as row r of a 128 x 64 piece in the
+// 128-byte-swizzled layout the TMA store expects (16-byte chunk j of row r sits at chunk
+// j ^ (r & 7)); consecutive rows hit different banks.
+__device__ __forceinline__ void stage_row_sw128(uint8_t* piece, int r, const uint32_t (&w)[32]) {
+  uint4* rowp = reinterpret_cast<uint4*>(piece + r * 128);
+#pragma unroll
+  for (int jc = 0; jc < 8; ++jc)
+    rowp[jc ^ (r & 7)] = make_uint4(w[4 * jc], w[4 * jc + 1], w[4 * jc + 2], w[4 * jc + 3]);
+}
+
+// AND-reduction of a predicate over the 128 epilogue threads (named barrier 1), so that
+// the decision to leave the tile loop is taken by all of them together.
+__device__ __forceinline__ bool epilogue_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok)
+      : "memory");
+  return r != 0;
+}
+
 template <int MODE, int A_MN, int B_MN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-            const GemmParams p) {
+            const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-  const uint32_t bar0 = base + kStages * kStageBytes;
+  uint8_t* out_smem = smem + kStages * kStageBytes;  // two 16 KB output pieces
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 2 * kOutBytes);
+  const uint32_t bar0 = base + kStages * kStageBytes + 2 * kOutBytes;
   // barrier slots: full[0..3], empty[4..7], tmem_full[8..9], tmem_empty[10..11]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
@@ -146,8 +196,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int n_live = (MODE == MODE_DEBUG) ? 0 : *p.n_live_ptr;
-  if (MODE != MODE_DEBUG && p.tag_ptr && *p.tag_ptr != kFwdTag) n_live = 0;
+  int row_begin = 0, row_end = 0;
+  if (MODE != MODE_DEBUG) {
+    int n_live = *p.n_live_ptr;
+    if (p.tag_ptr && *p.tag_ptr != kFwdTag) n_live = 0;
+    if (p.range_ptr) {
+      row_begin = p.range_ptr[0];
+      row_end = p.range_ptr[1];
+    } else {
+      row_begin = p.row_begin;
+      row_end = p.row_begin + p.row_cap;
+    }
+    if (row_end > n_live) row_end = n_live;
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -175,7 +236,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       Tile t;
       bool ok = true;
-      for (int j = 0; ok && get_tile<MODE>(p, n_live, j, t); ++j) {
+      for (int j = 0; ok && get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
         for (int kb = 0; kb < t.nk; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag)) {
@@ -209,7 +270,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       Tile t;
       bool ok = true;
-      for (int j = 0; ok && get_tile<MODE>(p, n_live, j, t); ++j) {
+      for (int j = 0; ok && get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
         const int buf = j & 1;
         if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
         tc_fence_after();
@@ -239,118 +300,160 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------ epilogue warps
     const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32)
     const int r_in_tile = quad * 32 + lane;
-    // MODE_LSE running state of this thread's row (log2 domain for the max)
+    const bool issuer = (threadIdx.x == 64);  // issues the TMA stores of the bf16 pieces
+    // running state of this thread's row across the tiles of a sweep
     float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f;
     Tile t;
-    for (int j = 0; get_tile<MODE>(p, n_live, j, t); ++j) {
+    for (int j = 0; get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
       const int buf = j & 1;
-      // per-row constants
-      const int row = t.m0 + r_in_tile;  // MODE_LSE/GRAD: compacted row; DH: chunk row; DW: vocab row
+      // MODE_LSE/GRAD/LSE_E: compacted row; DH: row inside the staged chunk; DW: vocabulary row
+      const int row = t.m0 + r_in_tile;
       int tgt = -1;
-      float cf = 0.f, lse2 = 0.f;
+      float cf = 0.f, ref2 = 0.f;
       bool valid = true;
-      if (MODE == MODE_LSE) {
-        valid = row < n_live;
+      if (MODE == MODE_LSE || MODE == MODE_LSE_E) {
+        valid = row < row_end;
         tgt = valid ? p.tgt_c[row] : -1;
+        if (MODE == MODE_LSE_E && valid) ref2 = p.zref[row] * kLog2e;
         if (t.first) { run_m2 = -INFINITY; run_l = 0.f; run_z = 0.f; }
       } else if (MODE == MODE_GRAD) {
-        valid = row < n_live;
+        valid = row < row_end;
         if (valid) {
           tgt = p.tgt_c[row];
           cf = p.coef[p.seq_c[row]];
-          lse2 = p.lse[row] * kLog2e;
+          ref2 = p.lse[row] * kLog2e;
         }
       }
-      if (!mbar_wait(tfull_bar(buf), (j >> 1) & 1u, abort_flag)) break;
+      const bool got = mbar_wait(tfull_bar(buf), (j >> 1) & 1u, abort_flag);
+      if (!epilogue_all(got)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;
+
+      if (MODE == MODE_GRAD || MODE == MODE_LSE_E) {
+        // bf16 output tile, 64 columns at a time: registers -> swizzled smem piece -> TMA store
 #pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c * 32, r);
-        tmem_ld_wait();
-        const int col0 = t.n0 + c * 32;
-        if (MODE == MODE_LSE) {
-          if (col0 < p.V) {
-            float v[32];
+        for (int g = 0; g < kBN / 64; ++g) {
+          uint32_t w[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-            if (col0 + 32 > p.V) {
+          for (int h = 0; h < 2; ++h) {
+            uint32_t r[32];
+            tmem_ld32(taddr + g * 64 + h * 32, r);
+            tmem_ld_wait();
+            const int col0 = t.n0 + g * 64 + h * 32;
+            if (valid && col0 < p.V) {
+              const int ti = tgt - col0;
+              if (MODE == MODE_LSE_E) {
+                float acc = 0.f;
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (col0 + i >= p.V) v[i] = -INFINITY;
-            }
-            float cmax = v[0];
+                for (int i = 0; i < 32; i += 2) {
+                  float e0 = ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -ref2));
+                  float e1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -ref2));
+                  if (col0 + i >= p.V) e0 = 0.f;
+                  if (col0 + i + 1 >= p.V) e1 = 0.f;
+                  acc += e0 + e1;
+                  w[h * 16 + (i >> 1)] = pack_bf16x2(e0, e1);
+                }
+                run_l += acc;
+                if (ti >= 0 && ti < 32) {
 #pragma unroll
-            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
-            const float m2 = fmaxf(run_m2, cmax * kLog2e);
-            float acc = 0.f;
+                  for (int i = 0; i < 32; ++i)
+                    if (i == ti) run_z = __uint_as_float(r[i]);
+                }
+              } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) acc += ex2_approx(fmaf(v[i], kLog2e, -m2));
-            run_l = run_l * ex2_approx(run_m2 - m2) + acc;
-            run_m2 = m2;
-            const int ti = tgt - col0;
-            if (ti >= 0 && ti < 32) {
+                for (int i = 0; i < 32; i += 2) {
+                  float g0 = -cf * ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -ref2));
+                  float g1 = -cf * ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -ref2));
+                  if (i == ti) g0 += cf;
+                  if (i + 1 == ti) g1 += cf;
+                  if (col0 + i >= p.V) g0 = 0.f;
+                  if (col0 + i + 1 >= p.V) g1 = 0.f;
+                  w[h * 16 + (i >> 1)] = pack_bf16x2(g0, g1);
+                }
+              }
+            } else {
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (i == ti) run_z = v[i];
+              for (int i = 0; i < 16; ++i) w[h * 16 + i] = 0u;
             }
           }
-        } else if (MODE == MODE_GRAD) {
-          uint32_t o[16];
-          if (valid && col0 < p.V) {
-            const int ti = tgt - col0;
+          uint8_t* piece = out_smem + (g & 1) * kOutBytes;
+          // the store that last read this piece (two pieces ago) must have drained it
+          if (issuer) tma_store_wait_read<1>();
+          epilogue_bar_sync();
+          stage_row_sw128(piece, r_in_tile, w);
+          fence_proxy_async_smem();
+          epilogue_bar_sync();
+          if (issuer) {
+            tma_store_2d(&tmC, smem_u32(piece), t.n0 + g * 64, t.m0 - row_begin);
+            tma_store_commit();
+          }
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c * 32, r);
+          tmem_ld_wait();
+          const int col0 = t.n0 + c * 32;
+          if (MODE == MODE_LSE) {
+            if (col0 < p.V) {
+              float v[32];
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              float g0 = -cf * ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -lse2));
-              float g1 = -cf * ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -lse2));
-              if (i == ti) g0 += cf;
-              if (i + 1 == ti) g1 += cf;
-              if (col0 + i >= p.V) g0 = 0.f;
-              if (col0 + i + 1 >= p.V) g1 = 0.f;
-              o[i >> 1] = pack_bf16x2(g0, g1);
+              for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+              if (col0 + 32 > p.V) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (col0 + i >= p.V) v[i] = -INFINITY;
+              }
+              float cmax = v[0];
+#pragma unroll
+              for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+              const float m2 = fmaxf(run_m2, cmax * kLog2e);
+              float acc = 0.f;
+#pragma unroll
+              for (int i = 0; i < 32; ++i) acc += ex2_approx(fmaf(v[i], kLog2e, -m2));
+              run_l = run_l * ex2_approx(run_m2 - m2) + acc;
+              run_m2 = m2;
+              const int ti = tgt - col0;
+              if (ti >= 0 && ti < 32) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (i == ti) run_z = v[i];
+              }
+            }
+          } else if (MODE == MODE_DH) {
+            const int crow = row_begin + row;
+            if (crow < row_end && col0 < p.d) {
+              const float sc = p.rowscale ? p.rowscale[crow] : 1.f;
+              uint32_t o[16];
+#pragma unroll
+              for (int i = 0; i < 32; i += 2)
+                o[i >> 1] = pack_bf16x2(sc * __uint_as_float(r[i]), sc * __uint_as_float(r[i + 1]));
+              uint4* dst = reinterpret_cast<uint4*>(p.dH + (size_t)p.live_rows[crow] * p.d + col0);
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+                dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+            }
+          } else if (MODE == MODE_DW) {
+            if (row < p.V && col0 < p.d) {
+              float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)row * p.d + col0);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {
+                float4 x = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                       __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+                if (p.accumulate) {
+                  const float4 y = dst[q];
+                  x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+                }
+                dst[q] = x;
+              }
             }
           } else {
+            if (row < p.M) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o[i] = 0u;
-          }
-          if (col0 < p.ldg) {
-            uint4* dst = reinterpret_cast<uint4*>(p.G + (size_t)(row - p.row_begin) * p.ldg + col0);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
-          }
-        } else if (MODE == MODE_DH) {
-          const int crow = p.row_begin + row;
-          if (crow < n_live && row < p.row_cap && col0 < p.d) {
-            uint32_t o[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 2)
-              o[i >> 1] = pack_bf16x2(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-            uint4* dst = reinterpret_cast<uint4*>(p.dH + (size_t)p.live_rows[crow] * p.d + col0);
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-              dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
-          }
-        } else if (MODE == MODE_DW) {
-          if (row < p.V && col0 < p.d) {
-            float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)row * p.d + col0);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float4 x = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                     __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
-              if (p.accumulate) {
-                const float4 y = dst[q];
-                x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
-              }
-              dst[q] = x;
+              for (int i = 0; i < 32; ++i)
+                if (col0 + i < p.N) p.Cdbg[(size_t)row * p.N + col0 + i] = __uint_as_float(r[i]);
             }
-          }
-        } else {
-          if (row < p.M) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (col0 + i < p.N) p.Cdbg[(size_t)row * p.N + col0 + i] = __uint_as_float(r[i]);
           }
         }
       }
@@ -358,15 +461,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
-      if (MODE == MODE_LSE) {
+      if (MODE == MODE_LSE || MODE == MODE_LSE_E) {
         if (t.last && valid) {
-          const size_t o = (size_t)row * p.C + t.split;
-          p.pm[o] = run_m2 * 0.6931471805599453f;  // back to natural units
+          const size_t o = (size_t)row * kMaxSplits + t.split;
+          if (MODE == MODE_LSE) p.pm[o] = run_m2 * kLn2;  // back to natural units
           p.pl[o] = run_l;
           p.pz[o] = run_z;
         }
       }
     }
+    if (issuer && (MODE == MODE_GRAD || MODE == MODE_LSE_E)) tma_store_wait_all();
   }
 
   // ---------------------------------------------------------------- teardown

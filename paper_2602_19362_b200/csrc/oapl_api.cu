@@ -18,15 +18,16 @@ namespace oapl {
 static std::atomic<uint64_t> g_launches{0};
 #define OAPL_LAUNCHED() (g_launches.fetch_add(1, std::memory_order_relaxed))
 
-constexpr int kMaxSplits = 16;
 constexpr int kChunkRowsDefault = 74 * 128;  // half of a 148-SM wave of row blocks
+constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref) in the single-call path
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Carve {
   size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, pm, pl, pz, cstart,
-      cend, seq_D, coef, vhat, seq_logp, Hc, G, total;
+      cend, seq_D, coef, vhat, seq_logp, Hc, G, zref, alpha, ztc, rowscale, Hs, ranges, total;
   int n_pad, nblk, chunk_rows, ldg;
+  int stage_rows, stage_alloc_rows, max_ranges;  // single-call path only
 };
 
 static int env_int(const char* name, int dflt) {
@@ -34,7 +35,7 @@ static int env_int(const char* name, int dflt) {
   return (s && *s) ? atoi(s) : dflt;
 }
 
-static bool carve(const oapl_problem* p, Carve* c) {
+static bool carve(const oapl_problem* p, int flags, Carve* c) {
   if (!p || p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return false;
   if (p->d % 64 != 0) return false;
   if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000) return false;
@@ -71,7 +72,26 @@ static bool carve(const oapl_problem* p, Carve* c) {
   c->vhat = take(4 * (size_t)p->P);
   c->seq_logp = take(4 * (size_t)p->S);
   c->Hc = take(2 * n_pad * (size_t)p->d);
-  c->G = take(2 * (size_t)chunk * (size_t)c->ldg);
+  c->stage_rows = c->stage_alloc_rows = c->max_ranges = 0;
+  if (flags & OAPL_FLAG_FUSED) {
+    // the chunk region holds e for a range of whole sequences instead of a row chunk of g
+    int stage = env_int("OAPL_STAGE_ROWS", kStageRowsDefault);
+    stage = (int)align_up((size_t)(stage < 128 ? 128 : stage), 128);
+    if ((size_t)stage > n_pad) stage = (int)n_pad;
+    c->stage_rows = stage;
+    c->stage_alloc_rows = stage + 128;
+    c->max_ranges = (int)(2 * n_pad / (size_t)stage) + 2;
+    c->G = take(2 * (size_t)c->stage_alloc_rows * (size_t)c->ldg);
+    c->zref = take(4 * n_pad);
+    c->alpha = take(4 * n_pad);
+    c->ztc = take(4 * n_pad);
+    c->rowscale = take(4 * n_pad);
+    c->Hs = take(2 * (n_pad + 128) * (size_t)p->d);
+    c->ranges = take(sizeof(RangeRec) * (size_t)c->max_ranges);
+  } else {
+    c->G = take(2 * (size_t)chunk * (size_t)c->ldg);
+    c->zref = c->alpha = c->ztc = c->rowscale = c->Hs = c->ranges = 0;
+  }
   c->total = off;
   return true;
 }
@@ -160,8 +180,8 @@ static void prof_end(int slot, cudaStream_t st) {
 }
 
 template <int MODE, int A_MN, int B_MN>
-static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmParams& gp, int grid,
-                       cudaStream_t st) {
+static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
+                       const GemmParams& gp, int grid, cudaStream_t st) {
   static bool attr_set = false;
   auto kern = gemm_kernel<MODE, A_MN, B_MN>;
   if (!attr_set) {
@@ -171,7 +191,7 @@ static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const GemmPar
     attr_set = true;
   }
   const int slot = prof_begin(MODE, st);
-  kern<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(a, b, gp);
+  kern<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(a, b, c, gp);
   OAPL_LAUNCHED();
   prof_end(slot, st);
   return cudaGetLastError() == cudaSuccess ? OAPL_OK : OAPL_ERR_CUDA;
@@ -204,9 +224,10 @@ static int check_problem(const oapl_problem* p, bool need_loss_inputs) {
     if (cudaGetLastError() != cudaSuccess) return OAPL_ERR_CUDA; \
   } while (0)
 
-// Shared forward: compaction, fused logits + online log-sum-exp, merge, per-sequence sums.
-static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, float* token_logp,
-                          float* seq_logp, bool with_q, cudaStream_t st) {
+// Live-row compaction shared by every forward: state word, compacted per-row arrays,
+// compacted-sequence bounds and the dense copy of the live rows of H.
+static int prologue(const oapl_problem* p, const Carve& c, uint8_t* ws, float* token_logp, bool with_q,
+                    cudaStream_t st) {
   const int n_sm = sm_count();
   if (n_sm <= 0) return OAPL_ERR_CUDA;
   DevState* state = reinterpret_cast<DevState*>(ws + c.state);
@@ -216,8 +237,6 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   int* tgt_c = reinterpret_cast<int*>(ws + c.tgt_c);
   int* seq_c = reinterpret_cast<int*>(ws + c.seq_c);
   float* q_c = reinterpret_cast<float*>(ws + c.q_c);
-  float* lp_c = reinterpret_cast<float*>(ws + c.lp_c);
-  float* lse = reinterpret_cast<float*>(ws + c.lse);
   int* cstart = reinterpret_cast<int*>(ws + c.cstart);
   int* cend = reinterpret_cast<int*>(ws + c.cend);
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + c.Hc);
@@ -241,6 +260,25 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gather_rows_kernel<<<n_sm * 8, 256, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(p->H), live_rows,
                                                state, p->d, Hc);
   CKL();
+  return OAPL_OK;
+}
+
+// Shared forward: compaction, fused logits + online log-sum-exp, merge, per-sequence sums.
+static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, float* token_logp,
+                          float* seq_logp, bool with_q, cudaStream_t st) {
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  int rc0 = prologue(p, c, ws, token_logp, with_q, st);
+  if (rc0 != OAPL_OK) return rc0;
+  DevState* state = reinterpret_cast<DevState*>(ws + c.state);
+  int* live_rows = reinterpret_cast<int*>(ws + c.live_rows);
+  int* tgt_c = reinterpret_cast<int*>(ws + c.tgt_c);
+  float* q_c = reinterpret_cast<float*>(ws + c.q_c);
+  float* lp_c = reinterpret_cast<float*>(ws + c.lp_c);
+  float* lse = reinterpret_cast<float*>(ws + c.lse);
+  int* cstart = reinterpret_cast<int*>(ws + c.cstart);
+  int* cend = reinterpret_cast<int*>(ws + c.cend);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + c.Hc);
 
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128)) return OAPL_ERR_CUDA;
@@ -258,14 +296,14 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.pz = reinterpret_cast<float*>(ws + c.pz);
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
-  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, gp, gp.R * gp.C, st);
+  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
-  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.C, state, live_rows, lse, lp_c,
-                                             token_logp);
+  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.R, gp.C, (p->V + kBN - 1) / kBN, state,
+                                             live_rows, lse, lp_c, token_logp);
   CKL();
   seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp,
-                                        reinterpret_cast<float*>(ws + c.seq_D), with_q ? 1 : 0);
+                                        reinterpret_cast<float*>(ws + c.seq_D), with_q ? 1 : 0, nullptr);
   CKL();
   return OAPL_OK;
 }
@@ -276,9 +314,9 @@ using namespace oapl;
 
 extern "C" {
 
-size_t oapl_workspace_bytes(const oapl_problem* problem, int /*flags*/) {
+size_t oapl_workspace_bytes(const oapl_problem* problem, int flags) {
   Carve c;
-  if (!carve(problem, &c)) return 0;
+  if (!carve(problem, flags, &c)) return 0;
   return c.total;
 }
 
@@ -295,6 +333,7 @@ const char* oapl_status_string(int status) {
     case OAPL_ERR_DEVICE_TIMEOUT: return "device pipeline wait timed out";
     case OAPL_ERR_CUDA: return "CUDA call failed";
     case OAPL_ERR_BAD_STATE: return "backward called without a matching forward";
+    case OAPL_ERR_SEQUENCE_TOO_LONG: return "a sequence has more live rows than the staging capacity";
     default: return "unknown status";
   }
 }
@@ -338,7 +377,7 @@ int oapl_token_logprobs(const oapl_problem* p, float* token_logp, float* seq_log
   if (!token_logp || !ws) return OAPL_ERR_INVALID_ARG;
   if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
   Carve c;
-  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (!carve(p, 0, &c)) return OAPL_ERR_INVALID_ARG;
   if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
   return forward_common(p, c, static_cast<uint8_t*>(ws), token_logp, seq_logp, false,
                         static_cast<cudaStream_t>(stream));
@@ -351,7 +390,7 @@ int oapl_loss_fwd(const oapl_problem* p, float* loss, float* seq_logp, float* vh
   if (!loss || !seq_logp || !vhat || !ws) return OAPL_ERR_INVALID_ARG;
   if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
   Carve c;
-  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (!carve(p, 0, &c)) return OAPL_ERR_INVALID_ARG;
   if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
   uint8_t* w = static_cast<uint8_t*>(ws);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -376,7 +415,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   if (((uintptr_t)dH | (uintptr_t)dW) & 15) return OAPL_ERR_MISALIGNED;
   if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
   Carve c;
-  if (!carve(p, &c)) return OAPL_ERR_INVALID_ARG;
+  if (!carve(p, 0, &c)) return OAPL_ERR_INVALID_ARG;
   if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
   const int n_sm = sm_count();
   if (n_sm <= 0) return OAPL_ERR_CUDA;
@@ -412,7 +451,6 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   gp.seq_c = reinterpret_cast<int*>(w + c.seq_c);
   gp.lse = reinterpret_cast<float*>(w + c.lse);
   gp.coef = reinterpret_cast<float*>(w + c.coef);
-  gp.G = G;
   gp.live_rows = reinterpret_cast<int*>(w + c.live_rows);
   gp.dH = static_cast<__nv_bfloat16*>(dH);
   gp.dW = dW;
@@ -425,13 +463,125 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   // find no tile and return at once.
   for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
     gp.row_begin = r0;
-    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, gp, gp.R * gp.C, st);
+    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, gp, n_sm, st);
+    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, tmGk, gp, n_sm, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, gp, n_sm, st);
+    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, tmGmn, gp, n_sm, st);
     if (rc != OAPL_OK) return rc;
   }
+  return OAPL_OK;
+}
+
+int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float* vhat, float* delta,
+                      float* token_logp, void* dH, float* dW, int accumulate_dW, void* ws,
+                      size_t ws_bytes, int flags, void* stream) {
+  int rc = check_problem(p, true);
+  if (rc != OAPL_OK) return rc;
+  if (!loss || !seq_logp || !vhat || !dH || !dW || !ws) return OAPL_ERR_INVALID_ARG;
+  if (((uintptr_t)dH | (uintptr_t)dW) & 15) return OAPL_ERR_MISALIGNED;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, flags | OAPL_FLAG_FUSED, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  rc = prologue(p, c, w, token_logp, true, st);
+  if (rc != OAPL_OK) return rc;
+  DevState* state = reinterpret_cast<DevState*>(w + c.state);
+  int* live_rows = reinterpret_cast<int*>(w + c.live_rows);
+  int* tgt_c = reinterpret_cast<int*>(w + c.tgt_c);
+  int* seq_c = reinterpret_cast<int*>(w + c.seq_c);
+  float* q_c = reinterpret_cast<float*>(w + c.q_c);
+  float* lp_c = reinterpret_cast<float*>(w + c.lp_c);
+  float* lse = reinterpret_cast<float*>(w + c.lse);
+  int* cstart = reinterpret_cast<int*>(w + c.cstart);
+  int* cend = reinterpret_cast<int*>(w + c.cend);
+  float* seq_D = reinterpret_cast<float*>(w + c.seq_D);
+  float* coef = reinterpret_cast<float*>(w + c.coef);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(w + c.Hc);
+  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(w + c.G);
+  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(w + c.Hs);
+  float* zref = reinterpret_cast<float*>(w + c.zref);
+  float* alpha = reinterpret_cast<float*>(w + c.alpha);
+  float* ztc = reinterpret_cast<float*>(w + c.ztc);
+  float* rowscale = reinterpret_cast<float*>(w + c.rowscale);
+  RangeRec* ranges = reinterpret_cast<RangeRec*>(w + c.ranges);
+  const int vtiles = (p->V + kBN - 1) / kBN;
+
+  CK(cudaMemsetAsync(seq_D, 0, 4 * (size_t)p->S, st));
+  CK(cudaMemsetAsync(seq_logp, 0, 4 * (size_t)p->S, st));
+  if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
+  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH),
+                                                  nullptr);
+  CKL();
+  value_estimate_kernel<<<(p->P + 7) / 8, 256, 0, st>>>(p->reward, p->group_id, p->S, p->P, p->beta_v,
+                                                        vhat, &state->status);
+  CKL();
+  ztgt_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, reinterpret_cast<const __nv_bfloat16*>(p->W), tgt_c, state,
+                                        p->d, p->V, zref);
+  CKL();
+  plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, c.max_ranges, ranges, state);
+  CKL();
+
+  CUtensorMap tmH, tmW, tmEk, tmWmn, tmEmn, tmHsmn;
+  const uint64_t ldg = (uint64_t)c.ldg;
+  bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
+            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256) &&
+            make_map(&tmEk, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 128) &&
+            make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
+            make_map(&tmEmn, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 64) &&
+            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 128, (uint64_t)p->d, (uint64_t)p->d, 64);
+  if (!ok) return OAPL_ERR_CUDA;
+
+  GemmParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.n_live_ptr = &state->n_live;
+  gp.d = p->d;
+  gp.V = p->V;
+  gp.ldg = c.ldg;
+  gp.pl = reinterpret_cast<float*>(w + c.pl);
+  gp.pz = reinterpret_cast<float*>(w + c.pz);
+  gp.tgt_c = tgt_c;
+  gp.zref = zref;
+  gp.live_rows = live_rows;
+  gp.dH = static_cast<__nv_bfloat16*>(dH);
+  gp.dW = dW;
+  gp.accumulate = 1;
+  gp.err = &state->status;
+  pick_sweep(n_sm, p->d, c.stage_rows / 128, vtiles, &gp.R, &gp.C);
+
+  // The ranges live on the device; the host enqueues the largest number of ranges the
+  // packing can produce and launches past the last range find no work.
+  for (int k = 0; k < c.max_ranges; ++k) {
+    const RangeRec* rg = ranges + k;
+    gp.range_ptr = &rg->row_begin;
+    gp.rowscale = nullptr;
+    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, gp.R * gp.C, st);
+    if (rc != OAPL_OK) return rc;
+    merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
+                                         alpha, ztc, token_logp);
+    CKL();
+    seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp, seq_D, 1, &rg->seq_begin);
+    CKL();
+    coef_range_kernel<<<(p->S + 255) / 256, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, rg, p->P,
+                                                          p->beta_loss, p->loss_scale, coef);
+    CKL();
+    scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, alpha, lse, ztc, rg, p->d, p->V,
+                                                 c.ldg, Hs, rowscale, E);
+    CKL();
+    rc = launch_gemm<MODE_DW, 1, 1>(tmEmn, tmHsmn, tmEmn, gp, n_sm, st);
+    if (rc != OAPL_OK) return rc;
+    gp.rowscale = rowscale;
+    rc = launch_gemm<MODE_DH, 0, 1>(tmEk, tmWmn, tmEk, gp, n_sm, st);
+    if (rc != OAPL_OK) return rc;
+  }
+  loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, p->S, p->P, p->beta_loss,
+                                 p->loss_scale, coef, delta, loss, state);
+  CKL();
   return OAPL_OK;
 }
 
@@ -482,10 +632,10 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
   const int grid = tiles < n_sm ? tiles : n_sm;
-  if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0>(ta, tb, gp, grid, st);
-  if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1>(ta, tb, gp, grid, st);
-  if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0>(ta, tb, gp, grid, st);
-  return launch_gemm<MODE_DEBUG, 1, 1>(ta, tb, gp, grid, st);
+  if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0>(ta, tb, ta, gp, grid, st);
+  if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1>(ta, tb, ta, gp, grid, st);
+  if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0>(ta, tb, ta, gp, grid, st);
+  return launch_gemm<MODE_DEBUG, 1, 1>(ta, tb, ta, gp, grid, st);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "sweep_schedule.cuh"
+
 namespace oapl {
 
 constexpr int kScanBlock = 1024;
@@ -146,7 +148,7 @@ __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ H, const in
 // ---- zero the dH rows of masked positions -------------------------------------------
 __global__ void zero_dead_rows_kernel(const uint8_t* __restrict__ mask, long long N, int d,
                                       __nv_bfloat16* __restrict__ dH, DevState* st) {
-  if (blockIdx.x == 0 && threadIdx.x == 0 && st->fwd_tag != 0x0A91) set_error(&st->status, -10);
+  if (st && blockIdx.x == 0 && threadIdx.x == 0 && st->fwd_tag != 0x0A91) set_error(&st->status, -10);
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int vec = d >> 3;
@@ -160,18 +162,23 @@ __global__ void zero_dead_rows_kernel(const uint8_t* __restrict__ mask, long lon
 }
 
 // ---- merge the per-split (max, sum-exp, target-logit) partials ----------------------
+// Row i has sweep_splits_of_block(...) partials in slots [i*kMaxSplits, ...).
 __global__ void merge_lse_kernel(const float* __restrict__ pm, const float* __restrict__ pl,
-                                 const float* __restrict__ pz, int C, const DevState* st,
-                                 const int* __restrict__ live_rows, float* __restrict__ lse,
-                                 float* __restrict__ lp_c, float* __restrict__ token_logp) {
+                                 const float* __restrict__ pz, int R, int C, int vtiles,
+                                 const DevState* st, const int* __restrict__ live_rows,
+                                 float* __restrict__ lse, float* __restrict__ lp_c,
+                                 float* __restrict__ token_logp) {
   const int n_live = st->n_live;
+  const int nrb = (n_live + 127) / 128;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_live; i += gridDim.x * blockDim.x) {
+    const int ns = sweep_splits_of_block(i / 128, nrb, R, C, vtiles);
+    const size_t o = (size_t)i * kMaxSplits;
     float M = -INFINITY;
-    for (int s = 0; s < C; ++s) M = fmaxf(M, pm[(size_t)i * C + s]);
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, pm[o + s]);
     float L = 0.f, z = 0.f;
-    for (int s = 0; s < C; ++s) {
-      L += pl[(size_t)i * C + s] * expf(pm[(size_t)i * C + s] - M);
-      z += pz[(size_t)i * C + s];
+    for (int s = 0; s < ns; ++s) {
+      L += pl[o + s] * expf(pm[o + s] - M);
+      z += pz[o + s];
     }
     const float l = M + logf(L);
     lse[i] = l;
@@ -190,9 +197,10 @@ __device__ __forceinline__ double warp_sum_d(double x) {
 __global__ void seq_sums_kernel(const float* __restrict__ lp_c, const float* __restrict__ q_c,
                                 const int* __restrict__ cstart, const int* __restrict__ cend,
                                 float* __restrict__ seq_logp, float* __restrict__ seq_D,
-                                int use_q) {
+                                int use_q, const int* __restrict__ seq_range) {
   __shared__ double sh[2][8];
   const int s = blockIdx.x;
+  if (seq_range && (s < seq_range[0] || s >= seq_range[1])) return;  // whole CTA
   const int b = cstart[s], e = cend[s];
   double a_lp = 0.0, a_df = 0.0;
   // scalar head up to a 16-byte boundary, float4 body, scalar tail
@@ -286,6 +294,165 @@ __global__ void loss_kernel(const float* __restrict__ reward, const int* __restr
     for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
     *loss = (float)((double)loss_scale * t);
     st->fwd_tag = 0x0A91;  // = kFwdTag of the contraction kernel
+  }
+}
+
+// =====================================================================================
+// Kernels of the single-call forward+backward path, which stages e = exp(z - zref) for a
+// range of whole sequences instead of recomputing the logits in the backward.
+// =====================================================================================
+struct RangeRec {
+  int row_begin, row_end;  // compacted rows
+  int seq_begin, seq_end;  // sequences whose live rows lie in the range (plus empty ones between)
+};
+
+// zref[i] = h_i . w_{y_i} + 40: a per-row reference close enough to the row's largest
+// logit that exp(z - zref) neither overflows (needs z_max - z_y < 128) nor loses the
+// dominant terms (z_max >= z_y, so they are >= e^-40).  One warp per live row.
+constexpr float kRefShift = 40.f;
+__global__ void ztgt_kernel(const __nv_bfloat16* __restrict__ Hc, const __nv_bfloat16* __restrict__ W,
+                            const int* __restrict__ tgt_c, const DevState* st, int d, int V,
+                            float* __restrict__ zref) {
+  const int n_live = st->n_live;
+  const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
+  for (int i = blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < n_live;
+       i += gridDim.x * warps_per_block) {
+    const int t = min(max(tgt_c[i], 0), V - 1);  // a bad target has already raised the error word
+    const uint4* h = reinterpret_cast<const uint4*>(Hc + (size_t)i * d);
+    const uint4* w = reinterpret_cast<const uint4*>(W + (size_t)t * d);
+    float acc = 0.f;
+    for (int k = lane; k < (d >> 3); k += 32) {
+      const uint4 a = h[k], b = __ldg(w + k);
+      const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+      const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 x = __bfloat1622float2(pa[q]), y = __bfloat1622float2(pb[q]);
+        acc = fmaf(x.x, y.x, acc);
+        acc = fmaf(x.y, y.y, acc);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) zref[i] = acc + kRefShift;
+  }
+}
+
+// Greedy packing of consecutive sequences into ranges of at most stage_rows live rows.
+// One thread; S is small.  Unused records are left empty.  A sequence longer than
+// stage_rows cannot be staged: the error word is raised and no range is produced.
+__global__ void plan_ranges_kernel(const int* __restrict__ cstart, const int* __restrict__ cend, int S,
+                                   int stage_rows, int max_ranges, RangeRec* __restrict__ ranges,
+                                   DevState* st) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
+  int n = 0, rb = -1, re = 0, sb = 0;
+  bool bad = false;
+  for (int s = 0; s < S && !bad; ++s) {
+    const int b = cstart[s], e = cend[s];
+    if (e <= b) continue;
+    if (e - b > stage_rows) { bad = true; break; }
+    if (rb < 0) { rb = b; sb = s; }
+    if (e - rb > stage_rows) {  // close the open range before this sequence
+      if (n < max_ranges) ranges[n] = RangeRec{rb, re, sb, s};
+      ++n;
+      rb = b;
+      sb = s;
+    }
+    re = e;
+  }
+  if (!bad && rb >= 0) {
+    if (n < max_ranges) ranges[n] = RangeRec{rb, re, sb, S};
+    ++n;
+  }
+  if (bad || n > max_ranges) {
+    for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
+    set_error(&st->status, bad ? -11 : -9);
+  }
+}
+
+// lse = zref + ln(sum_v e), token log-prob, and alpha = exp(zref - lse) = 1 / sum_v e.
+__global__ void merge_e_kernel(const float* __restrict__ pl, const float* __restrict__ pz,
+                               const float* __restrict__ zref, const RangeRec* __restrict__ range, int R,
+                               int C, int vtiles, const int* __restrict__ live_rows,
+                               float* __restrict__ lse, float* __restrict__ lp_c,
+                               float* __restrict__ alpha, float* __restrict__ ztc,
+                               float* __restrict__ token_logp) {
+  const int rb = range->row_begin, re = range->row_end;
+  const int nrb = (re - rb + 127) / 128;
+  for (int i = rb + blockIdx.x * blockDim.x + threadIdx.x; i < re; i += gridDim.x * blockDim.x) {
+    const int ns = sweep_splits_of_block((i - rb) / 128, nrb, R, C, vtiles);
+    const size_t o = (size_t)i * kMaxSplits;
+    float L = 0.f, z = 0.f;
+    for (int s = 0; s < ns; ++s) {
+      L += pl[o + s];
+      z += pz[o + s];
+    }
+    const float l = zref[i] + logf(L);
+    lse[i] = l;
+    ztc[i] = z;
+    alpha[i] = 1.f / L;
+    lp_c[i] = z - l;
+    if (token_logp) token_logp[live_rows[i]] = z - l;
+  }
+}
+
+// Coefficients c_i = 2 lambda beta_loss delta_i of the sequences of one range.
+__global__ void coef_range_kernel(const float* __restrict__ reward, const int* __restrict__ group_id,
+                                  const float* __restrict__ vhat, const float* __restrict__ seq_D,
+                                  const RangeRec* __restrict__ range, int P, float beta_loss,
+                                  float loss_scale, float* __restrict__ coef) {
+  for (int i = range->seq_begin + blockIdx.x * blockDim.x + threadIdx.x; i < range->seq_end;
+       i += gridDim.x * blockDim.x) {
+    const int g = group_id[i];
+    const float vh = (g >= 0 && g < P) ? vhat[g] : 0.f;
+    const double A = (double)reward[i] - (double)vh;
+    const double dl = (double)beta_loss * (double)seq_D[i] - A;
+    coef[i] = (float)(2.0 * (double)loss_scale * (double)beta_loss * dl);
+  }
+}
+
+// With s_n = -c_n * alpha_n:  g[n,v] = s_n * e'[n,v], where e' is e with the target entry
+// replaced by e_y - 1/alpha = (p_y - 1)/alpha.  So dH = rowscale(e'.W) and dW = e'^T.(s o H):
+// this kernel writes Hs = bf16(s_n H_n), the row scales, and patches the target entries.
+// Rows between the range end and the next multiple of 128 get zero Hs rows (the dW
+// contraction reads whole 64-row slabs).  One warp per row.
+__global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const int* __restrict__ seq_c,
+                                   const int* __restrict__ tgt_c, const float* __restrict__ coef,
+                                   const float* __restrict__ alpha, const float* __restrict__ lse,
+                                   const float* __restrict__ ztc, const RangeRec* __restrict__ range,
+                                   int d, int V, int ldg, __nv_bfloat16* __restrict__ Hs,
+                                   float* __restrict__ rowscale, __nv_bfloat16* __restrict__ E) {
+  const int rb = range->row_begin, re = range->row_end;
+  const int pad_end = rb + ((re - rb + 127) & ~127);
+  const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
+  const int vec = d >> 3;
+  for (int i = rb + blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < pad_end;
+       i += gridDim.x * warps_per_block) {
+    uint4* dst = reinterpret_cast<uint4*>(Hs + (size_t)i * d);
+    if (i < re) {
+      const float a = alpha[i];
+      const float s = -coef[seq_c[i]] * a;
+      const uint4* src = reinterpret_cast<const uint4*>(Hc + (size_t)i * d);
+      for (int k = lane; k < vec; k += 32) {
+        uint4 x = src[k];
+        __nv_bfloat162* px = reinterpret_cast<__nv_bfloat162*>(&x);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 f = __bfloat1622float2(px[q]);
+          px[q] = __floats2bfloat162_rn(s * f.x, s * f.y);
+        }
+        dst[k] = x;
+      }
+      if (lane == 0) {
+        rowscale[i] = s;
+        const int t = tgt_c[i];
+        if (t >= 0 && t < V)
+          E[(size_t)(i - rb) * ldg + t] = __float2bfloat16_rn(expm1f(ztc[i] - lse[i]) / a);
+      }
+    } else {
+      for (int k = lane; k < vec; k += 32) dst[k] = make_uint4(0, 0, 0, 0);
+    }
   }
 }
 

@@ -20,21 +20,30 @@ def npy(t):
     return t.detach().cpu().numpy()
 
 
-def run_gpu(dev, beta_v=None, beta_loss=None, loss_scale=None, backward=True, accumulate=False, dW_init=None):
+def run_gpu(dev, beta_v=None, beta_loss=None, loss_scale=None, backward=True, accumulate=False, dW_init=None,
+            fused=False):
+    """Run the CUDA path: oapl_loss_fwd (+ oapl_loss_bwd), or the single call
+    oapl_loss_fwd_bwd when fused=True."""
     prob = B.make_problem(dev, beta_v, beta_loss, loss_scale)
-    ws = B.alloc_workspace(prob)
+    ws = B.alloc_workspace(prob, B.OAPL_FLAG_FUSED if fused else 0)
     N, S, P, d, V = (dev[k] for k in ("N", "S", "P", "d", "V"))
     out = dict(loss=torch.full((1,), float("nan"), device="cuda"),
                seq_logp=torch.full((S,), float("nan"), device="cuda"),
                vhat=torch.full((P,), float("nan"), device="cuda"),
                delta=torch.full((S,), float("nan"), device="cuda"),
                token_logp=torch.full((N,), float("nan"), device="cuda"))
-    B.oapl_loss_fwd(prob, out["loss"], out["seq_logp"], out["vhat"], out["delta"], out["token_logp"], ws)
     if backward:
         out["dH"] = torch.full((N, d), float("nan"), dtype=torch.bfloat16, device="cuda")
         out["dW"] = (dW_init.clone() if dW_init is not None
                      else torch.full((V, d), float("nan"), dtype=torch.float32, device="cuda"))
-        B.oapl_loss_bwd(prob, out["dH"], out["dW"], accumulate, ws)
+    if fused:
+        assert backward
+        B.oapl_loss_fwd_bwd(prob, out["loss"], out["seq_logp"], out["vhat"], out["delta"], out["token_logp"],
+                            out["dH"], out["dW"], accumulate, ws)
+    else:
+        B.oapl_loss_fwd(prob, out["loss"], out["seq_logp"], out["vhat"], out["delta"], out["token_logp"], ws)
+        if backward:
+            B.oapl_loss_bwd(prob, out["dH"], out["dW"], accumulate, ws)
     out["status"] = B.oapl_get_last_status(ws)
     out["n_live"] = B.oapl_get_live_rows(ws)
     out["ws"] = ws

@@ -23,6 +23,8 @@ def test_small_variant_full_parity(name, rows):
     ref = hp.run_oracle(cpu, beta_v=betas[0], beta_loss=betas[0])
     mask = hp.npy(cpu["mask"])
     hp.assert_parity(out, ref, mask)
+    # the single-call path (no recompute) on the same inputs
+    hp.assert_parity(hp.run_gpu(dev, beta_v=betas[0], beta_loss=betas[0], fused=True), ref, mask)
     # remaining temperatures of the sweep: forward quantities only need the cached
     # oracle log-probs (Eq. 2 and Eq. 3 are O(S))
     for b in betas[1:]:

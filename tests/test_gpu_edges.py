@@ -12,9 +12,10 @@ pytestmark = pytest.mark.gpu
 TINY = synth.WORKLOADS["tiny"]
 
 
-def test_bitwise_run_to_run_determinism():
+@pytest.mark.parametrize("fused", [False, True], ids=["two-calls", "single-call"])
+def test_bitwise_run_to_run_determinism(fused):
     dev = hp.to_dev(synth.make_batch(TINY, seed=3))
-    a, b = hp.run_gpu(dev), hp.run_gpu(dev)
+    a, b = hp.run_gpu(dev, fused=fused), hp.run_gpu(dev, fused=fused)
     for k in ("loss", "seq_logp", "vhat", "delta", "token_logp", "dW"):
         assert torch.equal(a[k], b[k]), k
     assert torch.equal(a["dH"].view(torch.int16), b["dH"].view(torch.int16))
@@ -68,24 +69,26 @@ def test_degenerate_batches():
     cpu["mask"][cpu["seq_id"] == 5] = 0
     cpu["group_id"] = torch.tensor([0, 2, 1, 2, 0, 1, 2, 0, 1, 2, 0, 1, 2, 1, 0, 2], dtype=torch.int32)
     cpu["live_tokens"] = int(cpu["mask"].sum())
-    out = hp.run_gpu(hp.to_dev(cpu))
     ref = hp.run_oracle(cpu)
-    hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
-    assert float(out["seq_logp"][5]) == 0.0 and float(out["vhat"][3]) == 0.0
+    for fused in (False, True):
+        out = hp.run_gpu(hp.to_dev(cpu), fused=fused)
+        hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
+        assert float(out["seq_logp"][5]) == 0.0 and float(out["vhat"][3]) == 0.0
     # (b) nothing live at all: loss = lambda * sum A^2, gradients exactly zero
     cpu["mask"][:] = 0
-    out = hp.run_gpu(hp.to_dev(cpu))
     ref = hp.run_oracle(cpu)
-    assert out["status"] == 0 and out["n_live"] == 0
-    assert float(out["loss"]) == pytest.approx(ref["loss"], rel=1e-6)
-    assert float(out["dH"].float().abs().max()) == 0.0 and float(out["dW"].abs().max()) == 0.0
+    for fused in (False, True):
+        out = hp.run_gpu(hp.to_dev(cpu), fused=fused)
+        assert out["status"] == 0 and out["n_live"] == 0
+        assert float(out["loss"]) == pytest.approx(ref["loss"], rel=1e-6)
+        assert float(out["dH"].float().abs().max()) == 0.0 and float(out["dW"].abs().max()) == 0.0
     # (c) a single live row
     cpu["mask"][70] = 1
     cpu["targets"][70] = 17
     cpu["logp_inf"][70] = -8.0
-    out = hp.run_gpu(hp.to_dev(cpu))
     ref = hp.run_oracle(cpu)
-    hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
+    for fused in (False, True):
+        hp.assert_parity(hp.run_gpu(hp.to_dev(cpu), fused=fused), ref, hp.npy(cpu["mask"]))
 
 
 def test_one_token_vocab_and_all_equal_rewards():

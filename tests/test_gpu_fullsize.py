@@ -13,10 +13,11 @@ from tests import helpers as hp
 pytestmark = pytest.mark.gpu
 
 
-def test_7b_full_size_sampled_rows_and_invariants():
+@pytest.mark.parametrize("fused", [True, False], ids=["single-call", "two-calls"])
+def test_7b_full_size_sampled_rows_and_invariants(fused):
     wl = synth.WORKLOADS["7b"]
     dev = synth.make_batch(wl, seed=0, device="cuda", beta=1.0)
-    out = hp.run_gpu(dev)
+    out = hp.run_gpu(dev, fused=fused)
     assert out["status"] == 0 and out["n_live"] == dev["live_tokens"]
     N, S, P, d, V = (dev[k] for k in ("N", "S", "P", "d", "V"))
     mask = dev["mask"].bool()

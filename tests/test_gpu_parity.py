@@ -11,29 +11,35 @@ from tests import helpers as hp
 pytestmark = pytest.mark.gpu
 
 
-def _check(wl, seed=0, **kw):
+def _check(wl, seed=0, fused=False, **kw):
     cpu = synth.make_batch(wl, seed=seed)
-    out = hp.run_gpu(hp.to_dev(cpu), **kw)
+    out = hp.run_gpu(hp.to_dev(cpu), fused=fused, **kw)
     ref = hp.run_oracle(cpu, **kw)
     assert out["n_live"] == cpu["live_tokens"]
     hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
     return cpu, out, ref
 
 
-def test_tiny_config():
-    _check(synth.WORKLOADS["tiny"])
+BOTH = pytest.mark.parametrize("fused", [False, True], ids=["two-calls", "single-call"])
 
 
-def test_tiny_paper_temperatures_and_plain_sum():
+@BOTH
+def test_tiny_config(fused):
+    _check(synth.WORKLOADS["tiny"], fused=fused)
+
+
+@BOTH
+def test_tiny_paper_temperatures_and_plain_sum(fused):
     # beta_v = 1, beta_loss = 1e-3 (the paper's hyper-parameter tables), Eq. 3's plain sum
-    _check(synth.WORKLOADS["tiny"], seed=1, beta_v=1.0, beta_loss=1e-3, loss_scale=1.0)
+    _check(synth.WORKLOADS["tiny"], seed=1, beta_v=1.0, beta_loss=1e-3, loss_scale=1.0, fused=fused)
 
 
-def test_ragged_shapes():
+@BOTH
+def test_ragged_shapes(fused):
     # V not a multiple of the tile, d a multiple of 64 only, packed rows with masked prompt rows
     wl = dataclasses.replace(synth.small_variant("14b-long", prompts=3, samples=3, live_rows=700),
                              d=320, V=1000 + 37)
-    _check(wl, seed=2)
+    _check(wl, seed=2, fused=fused)
 
 
 def test_value_estimate_entry_point():
@@ -50,10 +56,27 @@ def test_value_estimate_entry_point():
         assert vhat[P - 1].item() == 0.0
 
 
-def test_many_chunks_and_waves_in_the_default_launch_configuration():
+@BOTH
+def test_many_chunks_and_waves_in_the_default_launch_configuration(fused):
     # about 20k response tokens: three default row chunks, several waves of row blocks
     # per chunk, sequences straddling tiles and chunks; small d and V keep the oracle fast
     wl = dataclasses.replace(synth.WORKLOADS["tiny"], prompts=16, samples=8, length=("uniform", 64, 256),
                              padded_to=256, d=256, V=4096 + 72)
-    cpu, out, ref = _check(wl, seed=11)
+    cpu, out, ref = _check(wl, seed=11, fused=fused)
     assert cpu["live_tokens"] > 2 * 9472
+
+
+def test_single_call_with_many_sequence_ranges(monkeypatch):
+    # a staging capacity of 512 rows forces ~40 ranges of whole sequences (lengths up to 256)
+    monkeypatch.setenv("OAPL_STAGE_ROWS", "512")
+    wl = dataclasses.replace(synth.WORKLOADS["tiny"], prompts=16, samples=8, length=("uniform", 64, 256),
+                             padded_to=256, d=256, V=4096 + 72)
+    _check(wl, seed=12, fused=True)
+
+
+def test_single_call_reports_a_sequence_longer_than_the_staging_capacity(monkeypatch):
+    monkeypatch.setenv("OAPL_STAGE_ROWS", "128")
+    wl = dataclasses.replace(synth.WORKLOADS["tiny"], length=("uniform", 150, 200), padded_to=256)
+    cpu = synth.make_batch(wl, seed=13)
+    out = hp.run_gpu(hp.to_dev(cpu), fused=True)
+    assert out["status"] == -11
