@@ -8,11 +8,16 @@
 //               sequences, per-row sum of e and target logit (no recompute in the backward)
 //   MODE_DEBUG  plain C = A.B for bring-up of the four operand-major combinations
 //
-// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM and issues the UMMAs,
-// warps 2..5 are the epilogue (one TMEM lane quadrant each).  Tile 128 x 256 x 64,
-// four shared-memory stages, two 256-column fp32 accumulators in TMEM so that the
-// epilogue of tile j overlaps the main loop of tile j+1.  bf16 tiles leave through
-// shared memory and TMA stores.
+// The kernel runs as pairs of CTAs (clusters of two, one pair per two SMs) that share
+// one 256 x 256 x 64 tile per step through tcgen05.mma.cta_group::2: each CTA loads its
+// own 128 rows of A and 128 of B's 256 columns (so every operand byte is fetched from L2
+// by one SM only, without multicast), the leader CTA's UMMA thread issues for both, and
+// each CTA's TMEM receives its 128 rows of the accumulator.
+// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM (and, in the leader, issues the
+// UMMAs), warps 2..5 are the epilogue (one TMEM lane quadrant each).  Six shared-memory
+// stages of 32 KB per CTA, two 256-column fp32 accumulators in TMEM so that the epilogue of
+// tile j overlaps the main loop of tile j+1.  bf16 tiles leave through shared memory and
+// TMA stores.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -24,9 +29,13 @@ namespace oapl {
 
 enum { MODE_LSE = 0, MODE_GRAD = 1, MODE_DH = 2, MODE_DW = 3, MODE_DEBUG = 4, MODE_LSE_E = 5 };
 
-constexpr int kBM = 128, kBN = 256, kBK = 64, kStages = 4;
-constexpr int kABytes = kBM * kBK * 2;  // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;  // 32 KB
+constexpr int kBM = 128;      // rows of A / of the accumulator per CTA
+constexpr int kTileM = 256;   // rows per CTA pair
+constexpr int kBN = 256;      // accumulator columns (per pair and per CTA)
+constexpr int kHalfN = 128;   // columns of B each CTA loads
+constexpr int kBK = 64, kStages = 6;
+constexpr int kABytes = kBM * kBK * 2;     // 16 KB
+constexpr int kBBytes = kHalfN * kBK * 2;  // 16 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kOutBytes = kBM * 64 * 2;  // one 128 x 64 bf16 output piece (16 KB), two of them
 constexpr int kGemmThreads = 192;
@@ -75,20 +84,22 @@ struct Tile {
   int first, last, split;
 };
 
-// Tile j of this CTA for rows [row_begin, row_end) of the compacted row space.
+// Tile j of this CTA pair for rows [row_begin, row_end) of the compacted row space.
+// m0 is the pair's first row; CTA `rank` of the pair owns rows m0 + 128*rank ....
 template <int MODE>
 __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int row_end, int j,
                                          Tile& t) {
   t.first = t.last = 1;
   t.split = 0;
   const int rows = row_end - row_begin;
+  const int pid = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
     if (rows <= 0) return false;
     const int VT = (p.V + kBN - 1) / kBN;
-    const int nrb = (rows + kBM - 1) / kBM;
+    const int nrb = (rows + kTileM - 1) / kTileM;
     const SweepShape sh = sweep_shape(nrb, p.R, p.C, VT);
     // complete waves: this CTA is (row block rbi, split s) of every wave
-    const int rbi = blockIdx.x % p.R, s = blockIdx.x / p.R;
+    const int rbi = pid % p.R, s = pid / p.R;
     int vt0 = (int)((long long)VT * s / p.C), vt1 = (int)((long long)VT * (s + 1) / p.C);
     int per = (s < p.C) ? vt1 - vt0 : 0;
     const int main_tiles = sh.nfull * per;
@@ -101,7 +112,7 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
     } else {
       // tail wave: rem row blocks x Ct splits
       if (sh.rem == 0) return false;
-      const int rbt = blockIdx.x % sh.rem, st = blockIdx.x / sh.rem;
+      const int rbt = pid % sh.rem, st = pid / sh.rem;
       if (st >= sh.Ct) return false;
       vt0 = (int)((long long)VT * st / sh.Ct);
       vt1 = (int)((long long)VT * (st + 1) / sh.Ct);
@@ -111,7 +122,7 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
       rbk = sh.nfull * p.R + rbt;
       t.split = st;
     }
-    t.m0 = row_begin + rbk * kBM;
+    t.m0 = row_begin + rbk * kTileM;
     t.n0 = (vt0 + off) * kBN;
     t.ka0 = t.kb0 = 0;
     t.nk = p.d / kBK;
@@ -120,30 +131,30 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
     return true;
   } else if (MODE == MODE_DH) {
     if (rows <= 0) return false;
-    const int MB = (rows + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
-    const int tix = blockIdx.x + j * gridDim.x;
+    const int MB = (rows + kTileM - 1) / kTileM, NB = (p.d + kBN - 1) / kBN;
+    const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kBM;  // row inside the staged chunk
+    t.m0 = (tix / NB) * kTileM;  // row inside the staged chunk
     t.n0 = (tix % NB) * kBN;
     t.ka0 = t.kb0 = 0;
     t.nk = (p.V + kBK - 1) / kBK;
     return true;
   } else if (MODE == MODE_DW) {
     if (rows <= 0) return false;
-    const int MB = (p.V + kBM - 1) / kBM, NB = (p.d + kBN - 1) / kBN;
-    const int tix = blockIdx.x + j * gridDim.x;
+    const int MB = (p.V + kTileM - 1) / kTileM, NB = (p.d + kBN - 1) / kBN;
+    const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kBM;  // vocabulary row
+    t.m0 = (tix / NB) * kTileM;  // vocabulary row
     t.n0 = (tix % NB) * kBN;
     t.ka0 = 0;          // staged chunk rows are range-relative
     t.kb0 = row_begin;  // compacted H rows are absolute
     t.nk = (rows + kBK - 1) / kBK;
     return true;
   } else {
-    const int MB = (p.M + kBM - 1) / kBM, NB = (p.N + kBN - 1) / kBN;
-    const int tix = blockIdx.x + j * gridDim.x;
+    const int MB = (p.M + kTileM - 1) / kTileM, NB = (p.N + kBN - 1) / kBN;
+    const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kBM;
+    t.m0 = (tix / NB) * kTileM;
     t.n0 = (tix % NB) * kBN;
     t.ka0 = t.kb0 = 0;
     t.nk = p.K / kBK;
@@ -177,7 +188,7 @@ __device__ __forceinline__ bool epilogue_all(bool ok) {
 }
 
 template <int MODE, int A_MN, int B_MN>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -196,6 +207,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStages + 5);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader of the pair
   int row_begin = 0, row_end = 0;
   if (MODE != MODE_DEBUG) {
     int n_live = *p.n_live_ptr;
@@ -217,7 +229,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 4);
+      mbar_init(tempty_bar(b), 8);  // leader's copy is used: 4 epilogue warps of each CTA
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -227,6 +239,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();  // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -244,29 +257,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
-          mbar_expect_tx(full_bar(s), kStageBytes);
+          // the leader's barrier collects the bytes of both CTAs' loads
+          const uint32_t fb = mapa_shared(full_bar(s), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes);
           const int ka = t.ka0 + kb * kBK, kbb = t.kb0 + kb * kBK;
+          const int am = t.m0 + (int)rank * kBM, bn = t.n0 + (int)rank * kHalfN;
           if (A_MN) {
 #pragma unroll
-            for (int b = 0; b < kBM / 64; ++b)
-              tma_load_2d(sa + b * 8192, &tmA, full_bar(s), t.m0 + 64 * b, ka);
+            for (int b = 0; b < kBM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, fb, am + 64 * b, ka);
           } else {
-            tma_load_2d(sa, &tmA, full_bar(s), ka, t.m0);
+            tma_load_2d(sa, &tmA, fb, ka, am);
           }
           if (B_MN) {
 #pragma unroll
-            for (int b = 0; b < kBN / 64; ++b)
-              tma_load_2d(sb + b * 8192, &tmB, full_bar(s), t.n0 + 64 * b, kbb);
+            for (int b = 0; b < kHalfN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, fb, bn + 64 * b, kbb);
           } else {
-            tma_load_2d(sb, &tmB, full_bar(s), kbb, t.n0);
+            tma_load_2d(sb, &tmB, fb, kbb, bn);
           }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(kBM, kBN, A_MN, B_MN);
+    // ------------------------------------------------------------ UMMA issuer (leader CTA only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(kTileM, kBN, A_MN, B_MN);
       uint32_t it = 0;
       Tile t;
       bool ok = true;
@@ -291,9 +305,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                      : smem_desc_sw128(sb + kk * 32, 16, 1024);
             umma_bf16(d_tmem, da, db, idesc, (kb | kk) ? 1u : 0u);
           }
-          umma_commit(empty_bar(s));  // stage reusable once these UMMAs have read it
+          umma_commit_pair(empty_bar(s));  // both CTAs' stage reusable once these UMMAs have read it
         }
-        if (ok) umma_commit(tfull_bar(buf));  // accumulator complete
+        if (ok) umma_commit_pair(tfull_bar(buf));  // accumulator complete in both CTAs
       }
     }
   } else {
@@ -307,7 +321,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     for (int j = 0; get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
       const int buf = j & 1;
       // MODE_LSE/GRAD/LSE_E: compacted row; DH: row inside the staged chunk; DW: vocabulary row
-      const int row = t.m0 + r_in_tile;
+      const int row = t.m0 + (int)rank * kBM + r_in_tile;
       int tgt = -1;
       float cf = 0.f, ref2 = 0.f;
       bool valid = true;
@@ -384,7 +398,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           fence_proxy_async_smem();
           epilogue_bar_sync();
           if (issuer) {
-            tma_store_2d(&tmC, smem_u32(piece), t.n0 + g * 64, t.m0 - row_begin);
+            tma_store_2d(&tmC, smem_u32(piece), t.n0 + g * 64, t.m0 - row_begin + (int)rank * kBM);
             tma_store_commit();
           }
         }
@@ -460,7 +474,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // accumulator drained: hand the TMEM buffer back to the UMMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
       if (MODE == MODE_LSE || MODE == MODE_LSE_E) {
         if (t.last && valid) {
           const size_t o = (size_t)row * kMaxSplits + t.split;
@@ -485,6 +499,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     __syncthreads();
   }
+  // neither CTA may release its TMEM or shared memory while the other can still touch them
+  cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);

@@ -39,11 +39,11 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
   if (!p || p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return false;
   if (p->d % 64 != 0) return false;
   if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000) return false;
-  const size_t n_pad = align_up((size_t)p->N, 128);
+  const size_t n_pad = align_up((size_t)p->N, 256);
   c->n_pad = (int)n_pad;
   c->nblk = (int)((p->N + kScanBlock - 1) / kScanBlock);
   int chunk = env_int("OAPL_CHUNK_ROWS", kChunkRowsDefault);
-  chunk = (int)align_up((size_t)(chunk < 128 ? 128 : chunk), 128);
+  chunk = (int)align_up((size_t)(chunk < 256 ? 256 : chunk), 256);
   if ((size_t)chunk > n_pad) chunk = (int)n_pad;
   c->chunk_rows = chunk;
   c->ldg = (int)align_up((size_t)p->V, 256);
@@ -76,17 +76,17 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
   if (flags & OAPL_FLAG_FUSED) {
     // the chunk region holds e for a range of whole sequences instead of a row chunk of g
     int stage = env_int("OAPL_STAGE_ROWS", kStageRowsDefault);
-    stage = (int)align_up((size_t)(stage < 128 ? 128 : stage), 128);
+    stage = (int)align_up((size_t)(stage < 256 ? 256 : stage), 256);
     if ((size_t)stage > n_pad) stage = (int)n_pad;
     c->stage_rows = stage;
-    c->stage_alloc_rows = stage + 128;
+    c->stage_alloc_rows = stage + 256;
     c->max_ranges = (int)(2 * n_pad / (size_t)stage) + 2;
     c->G = take(2 * (size_t)c->stage_alloc_rows * (size_t)c->ldg);
     c->zref = take(4 * n_pad);
     c->alpha = take(4 * n_pad);
     c->ztc = take(4 * n_pad);
     c->rowscale = take(4 * n_pad);
-    c->Hs = take(2 * (n_pad + 128) * (size_t)p->d);
+    c->Hs = take(2 * (n_pad + 256) * (size_t)p->d);
     c->ranges = take(sizeof(RangeRec) * (size_t)c->max_ranges);
   } else {
     c->G = take(2 * (size_t)chunk * (size_t)c->ldg);
@@ -139,22 +139,22 @@ static int sm_count() {
   return n;
 }
 
-// Sweep schedule: C vocabulary splits x R row blocks per wave, R*C <= SM count.  C is
-// the smallest power of two that keeps the wave's H row blocks within an L2 budget and
-// does not leave SMs without a row block when the row range is short.
-static void pick_sweep(int n_sm, int d, int rb_max, int vtiles, int* R, int* C) {
+// Sweep schedule: a wave is R row blocks (256 rows, one CTA pair each) x C vocabulary
+// splits, R*C <= number of CTA pairs.  C is the smallest power of two that keeps the wave's
+// H row blocks within an L2 budget; a short row range is handled by the tail-wave
+// re-splitting of the schedule itself.
+static void pick_sweep(int n_sm, int d, int vtiles, int* R, int* C) {
+  const int pairs = n_sm / 2;
   int c = env_int("OAPL_SPLITS", 0);
   if (c <= 0) {
     c = 1;
-    const size_t budget = (size_t)env_int("OAPL_L2_BUDGET_MB", 40) << 20;
-    while (c < kMaxSplits && (size_t)(n_sm / c) * 128 * d * 2 > budget) c *= 2;
-    while (c < kMaxSplits && n_sm / c > rb_max) c *= 2;
+    const size_t budget = (size_t)env_int("OAPL_L2_BUDGET_MB", 72) << 20;
+    while (c < kMaxSplits && (size_t)(pairs / c) * kSweepRows * d * 2 > budget) c *= 2;
   }
   if (c > kMaxSplits) c = kMaxSplits;
   while (c > 1 && c > vtiles) c /= 2;
-  int r = n_sm / c;
+  int r = pairs / c;
   if (r < 1) r = 1;
-  if (r > rb_max) r = rb_max;
   *R = r;
   *C = c;
 }
@@ -282,13 +282,13 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
 
   CUtensorMap tmA, tmB;
   if (!make_map(&tmA, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128)) return OAPL_ERR_CUDA;
-  if (!make_map(&tmB, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256)) return OAPL_ERR_CUDA;
+  if (!make_map(&tmB, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128)) return OAPL_ERR_CUDA;
   GemmParams gp;
   memset(&gp, 0, sizeof(gp));
   gp.n_live_ptr = &state->n_live;
   gp.row_begin = 0;
   gp.row_cap = c.n_pad;
-  pick_sweep(n_sm, p->d, c.n_pad / 128, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+  pick_sweep(n_sm, p->d, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
   gp.d = p->d;
   gp.V = p->V;
   gp.pm = reinterpret_cast<float*>(ws + c.pm);
@@ -296,7 +296,7 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.pz = reinterpret_cast<float*>(ws + c.pz);
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
-  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, gp.R * gp.C, st);
+  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
   merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.R, gp.C, (p->V + kBN - 1) / kBN, state,
@@ -432,7 +432,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   CUtensorMap tmH, tmW, tmGk, tmWmn, tmGmn, tmHmn;
   const uint64_t ldg = (uint64_t)c.ldg;
   bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
-            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256) &&
+            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmGk, G, (uint64_t)c.chunk_rows, ldg, ldg, 128) &&
             make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
             make_map(&tmGmn, G, (uint64_t)c.chunk_rows, ldg, ldg, 64) &&
@@ -456,18 +456,18 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   gp.dW = dW;
   gp.accumulate = 1;  // dW is zeroed above unless the caller accumulates; every chunk adds
   gp.err = &state->status;
-  pick_sweep(n_sm, p->d, c.chunk_rows / 128, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+  pick_sweep(n_sm, p->d, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
 
   // Row chunks of the compacted rows.  The live-row count lives on the device, so the
   // host enqueues every chunk the row count N could need; chunks past the live rows
   // find no tile and return at once.
   for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
     gp.row_begin = r0;
-    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, gp.R * gp.C, st);
+    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, tmGk, gp, n_sm, st);
+    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, tmGmn, gp, n_sm, st);
+    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, tmGmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
   return OAPL_OK;
@@ -530,11 +530,11 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   CUtensorMap tmH, tmW, tmEk, tmWmn, tmEmn, tmHsmn;
   const uint64_t ldg = (uint64_t)c.ldg;
   bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
-            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 256) &&
+            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmEk, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 128) &&
             make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
             make_map(&tmEmn, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 64) &&
-            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 128, (uint64_t)p->d, (uint64_t)p->d, 64);
+            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 256, (uint64_t)p->d, (uint64_t)p->d, 64);
   if (!ok) return OAPL_ERR_CUDA;
 
   GemmParams gp;
@@ -552,7 +552,7 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   gp.dW = dW;
   gp.accumulate = 1;
   gp.err = &state->status;
-  pick_sweep(n_sm, p->d, c.stage_rows / 128, vtiles, &gp.R, &gp.C);
+  pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
 
   // The ranges live on the device; the host enqueues the largest number of ranges the
   // packing can produce and launches past the last range find no work.
@@ -560,7 +560,7 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
     const RangeRec* rg = ranges + k;
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
-    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, gp.R * gp.C, st);
+    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
     merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
                                          alpha, ztc, token_logp);
@@ -573,10 +573,10 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
     scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, alpha, lse, ztc, rg, p->d, p->V,
                                                  c.ldg, Hs, rowscale, E);
     CKL();
-    rc = launch_gemm<MODE_DW, 1, 1>(tmEmn, tmHsmn, tmEmn, gp, n_sm, st);
+    rc = launch_gemm<MODE_DW, 1, 1>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
     gp.rowscale = rowscale;
-    rc = launch_gemm<MODE_DH, 0, 1>(tmEk, tmWmn, tmEk, gp, n_sm, st);
+    rc = launch_gemm<MODE_DH, 0, 1>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
   loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, p->S, p->P, p->beta_loss,
@@ -620,7 +620,7 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   bool ok = a_mn ? make_map(&ta, A, (uint64_t)K, (uint64_t)M, (uint64_t)M, 64)
                  : make_map(&ta, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128);
   ok = ok && (b_mn ? make_map(&tb, B, (uint64_t)K, (uint64_t)N, (uint64_t)N, 64)
-                   : make_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, 256));
+                   : make_map(&tb, B, (uint64_t)N, (uint64_t)K, (uint64_t)K, 128));
   if (!ok) return OAPL_ERR_CUDA;
   GemmParams gp;
   memset(&gp, 0, sizeof(gp));
@@ -630,8 +630,8 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   gp.K = K;
   gp.err = err;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
-  const int grid = tiles < n_sm ? tiles : n_sm;
+  const int tiles = ((M + kTileM - 1) / kTileM) * ((N + kBN - 1) / kBN);
+  const int grid = 2 * (tiles < n_sm / 2 ? tiles : n_sm / 2);
   if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0>(ta, tb, ta, gp, grid, st);
   if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1>(ta, tb, ta, gp, grid, st);
   if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0>(ta, tb, ta, gp, grid, st);
@@ -694,7 +694,7 @@ int oapl_token_logprobs_static(const oapl_problem* p, float* token_logp, float* 
   // Lay the forward's scratch out inside the fixed array (1 KB-aligned pieces).
   Carve c;
   memset(&c, 0, sizeof(c));
-  const size_t n_pad = align_up((size_t)p->N, 128);
+  const size_t n_pad = align_up((size_t)p->N, 256);
   c.n_pad = (int)n_pad;
   c.nblk = (int)((p->N + kScanBlock - 1) / kScanBlock);
   c.chunk_rows = (int)n_pad;

@@ -125,11 +125,11 @@ __global__ void seq_bounds_kernel(const int* __restrict__ seq_c, const DevState*
   }
 }
 
-// ---- gather live rows of H into a dense [round_up(n_live,128), d] matrix ----------
+// ---- gather live rows of H into a dense [round_up(n_live,256), d] matrix ----------
 __global__ void gather_rows_kernel(const __nv_bfloat16* __restrict__ H, const int* __restrict__ live_rows,
                                    const DevState* st, int d, __nv_bfloat16* __restrict__ Hc) {
   const int n_live = st->n_live;
-  const int n_pad = (n_live + 127) & ~127;
+  const int n_pad = (n_live + 255) & ~255;
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   const int vec = d >> 3;  // uint4 per row
@@ -169,9 +169,9 @@ __global__ void merge_lse_kernel(const float* __restrict__ pm, const float* __re
                                  float* __restrict__ lse, float* __restrict__ lp_c,
                                  float* __restrict__ token_logp) {
   const int n_live = st->n_live;
-  const int nrb = (n_live + 127) / 128;
+  const int nrb = (n_live + kSweepRows - 1) / kSweepRows;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_live; i += gridDim.x * blockDim.x) {
-    const int ns = sweep_splits_of_block(i / 128, nrb, R, C, vtiles);
+    const int ns = sweep_splits_of_block(i / kSweepRows, nrb, R, C, vtiles);
     const size_t o = (size_t)i * kMaxSplits;
     float M = -INFINITY;
     for (int s = 0; s < ns; ++s) M = fmaxf(M, pm[o + s]);
@@ -379,9 +379,9 @@ __global__ void merge_e_kernel(const float* __restrict__ pl, const float* __rest
                                float* __restrict__ alpha, float* __restrict__ ztc,
                                float* __restrict__ token_logp) {
   const int rb = range->row_begin, re = range->row_end;
-  const int nrb = (re - rb + 127) / 128;
+  const int nrb = (re - rb + kSweepRows - 1) / kSweepRows;
   for (int i = rb + blockIdx.x * blockDim.x + threadIdx.x; i < re; i += gridDim.x * blockDim.x) {
-    const int ns = sweep_splits_of_block((i - rb) / 128, nrb, R, C, vtiles);
+    const int ns = sweep_splits_of_block((i - rb) / kSweepRows, nrb, R, C, vtiles);
     const size_t o = (size_t)i * kMaxSplits;
     float L = 0.f, z = 0.f;
     for (int s = 0; s < ns; ++s) {
@@ -415,7 +415,7 @@ __global__ void coef_range_kernel(const float* __restrict__ reward, const int* _
 // With s_n = -c_n * alpha_n:  g[n,v] = s_n * e'[n,v], where e' is e with the target entry
 // replaced by e_y - 1/alpha = (p_y - 1)/alpha.  So dH = rowscale(e'.W) and dW = e'^T.(s o H):
 // this kernel writes Hs = bf16(s_n H_n), the row scales, and patches the target entries.
-// Rows between the range end and the next multiple of 128 get zero Hs rows (the dW
+// Rows between the range end and the next multiple of 256 get zero Hs rows (the dW
 // contraction reads whole 64-row slabs).  One warp per row.
 __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const int* __restrict__ seq_c,
                                    const int* __restrict__ tgt_c, const float* __restrict__ coef,
@@ -424,7 +424,7 @@ __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const i
                                    int d, int V, int ldg, __nv_bfloat16* __restrict__ Hs,
                                    float* __restrict__ rowscale, __nv_bfloat16* __restrict__ E) {
   const int rb = range->row_begin, re = range->row_end;
-  const int pad_end = rb + ((re - rb + 127) & ~127);
+  const int pad_end = rb + ((re - rb + 255) & ~255);
   const int warps_per_block = blockDim.x >> 5, lane = threadIdx.x & 31;
   const int vec = d >> 3;
   for (int i = rb + blockIdx.x * warps_per_block + (threadIdx.x >> 5); i < pad_end;

@@ -1,9 +1,9 @@
 // Schedule of the vocabulary-sweep kernels, shared by the contraction kernel (which
 // walks it) and the merge kernels (which need to know how many partial results a row has).
 //
-// The rows of a range are cut into 128-row blocks.  A wave is R row blocks x C
-// vocabulary splits = R*C CTAs, each sweeping its split's vocabulary tiles for one row
-// block.  The last, incomplete wave (rem < R row blocks) is re-split into Ct >= C
+// The rows of a range are cut into 256-row blocks (one per CTA pair).  A wave is R row
+// blocks x C vocabulary splits = R*C CTA pairs, each sweeping its split's vocabulary tiles
+// for one row block.  The last, incomplete wave (rem < R row blocks) is re-split into Ct >= C
 // vocabulary splits so that it still occupies (almost) every CTA for a proportionally
 // shorter time instead of leaving most of them idle.
 #pragma once
@@ -11,6 +11,7 @@
 namespace oapl {
 
 constexpr int kMaxSplits = 16;
+constexpr int kSweepRows = 256;  // rows per row block of the sweep
 
 struct SweepShape {
   int nfull;  // complete waves

@@ -75,8 +75,8 @@ def test_single_call_with_many_sequence_ranges(monkeypatch):
 
 
 def test_single_call_reports_a_sequence_longer_than_the_staging_capacity(monkeypatch):
-    monkeypatch.setenv("OAPL_STAGE_ROWS", "128")
-    wl = dataclasses.replace(synth.WORKLOADS["tiny"], length=("uniform", 150, 200), padded_to=256)
+    monkeypatch.setenv("OAPL_STAGE_ROWS", "256")
+    wl = dataclasses.replace(synth.WORKLOADS["tiny"], length=("uniform", 300, 400), padded_to=512)
     cpu = synth.make_batch(wl, seed=13)
     out = hp.run_gpu(hp.to_dev(cpu), fused=True)
     assert out["status"] == -11
