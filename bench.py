@@ -251,6 +251,7 @@ def run_cuda(args) -> None:
     total_ms = ev[0].elapsed_time(ev[args.steps])
     step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
     prof = B.oapl_profile_read()
+    prof_mhz = B.oapl_profile_read_clocks()
     B.oapl_profile_enable(False)
     clocks = sampler.stop() if rank == 0 else None
     st = B.oapl_get_last_status(ws)
@@ -319,7 +320,8 @@ def run_cuda(args) -> None:
                 "credited_frac_of_burst": flops_step / (ms_step * 1e-3) / 1e12 / peaks["burst"],
                 "credited_frac_of_nominal_2250": flops_step / (ms_step * 1e-3) / 1e12 / 2250.0,
                 "contraction_ms_per_step": gemm_ms, "contraction_launches_per_step": gemm_launches,
-                "by_kind_ms_per_step": {k: v[0] / args.steps for k, v in prof.items() if v[1]}}
+                "by_kind_ms_per_step": {k: v[0] / args.steps for k, v in prof.items() if v[1]},
+                "by_kind_sm_mhz": {k: round(prof_mhz[k]) for k, v in prof.items() if v[1]}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",

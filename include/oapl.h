@@ -191,17 +191,27 @@ int oapl_token_logprobs_static(const oapl_problem* problem /*host*/, float* toke
  */
 int oapl_profile_enable(int on);
 int oapl_profile_read(float* ms_by_kind /*host*/, int* launches_by_kind /*host*/, int kinds);
+/*
+ * While the timing is enabled, CTA 0 of every contraction launch also adds its SM cycle count
+ * and its elapsed nanoseconds to two per-kind device counters.  This call synchronises the
+ * device, writes cycles/nanoseconds as MHz per kind (0 where the kind did not run) -- the SM
+ * clock that kind of launch ran at, which on a power-capped part differs from kind to kind --
+ * and clears the counters.  kinds <= 8.
+ */
+int oapl_profile_read_clocks(float* sm_mhz_by_kind /*host*/, int kinds);
 
 /*
  * Bring-up aid for the tensor-core main loop shared by every contraction above:
  * C[M, N] (f32 row-major, ld = N) = A . B with bf16 operands, through the same
  * TMA/tcgen05 pipeline.  a_mn == 0: A is [M, K] row-major (K contiguous);
  * a_mn == 1: A is stored [K, M] row-major (M contiguous).  b_mn == 0: B is stored
- * [N, K] row-major; b_mn == 1: B is stored [K, N] row-major.  K % 64 == 0,
- * M % 8 == 0, N % 8 == 0.  `err` is a device int the kernel sets on a timeout.
+ * [N, K] row-major; b_mn == 1: B is stored [K, N] row-major.  wide == 0: 256 x 256 tiles
+ * with alternating accumulators (the vocabulary sweeps' shape); wide == 1: 256 x 512 tiles
+ * (the shape of the dH and dW contractions).  K % 64 == 0, M % 8 == 0, N % 8 == 0.
+ * `err` is a device int the kernel sets on a timeout.
  */
 int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn,
-                    int b_mn, int* err, void* stream);
+                    int b_mn, int wide, int* err, void* stream);
 
 #ifdef __cplusplus
 }

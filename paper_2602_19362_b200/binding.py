@@ -22,7 +22,7 @@ OAPL_FLAG_FUSED = 1
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
-           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd"]
+           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -72,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.oapl_status_string.restype = ctypes.c_char_p
         L.oapl_status_string.argtypes = [i32]
         L.oapl_debug_gemm.restype = i32
-        L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+        L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
         L.oapl_loss_fwd_bwd.restype = i32
         L.oapl_loss_fwd_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_token_logprobs_static.restype = i32
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.oapl_profile_enable.argtypes = [i32]
         L.oapl_profile_read.restype = i32
         L.oapl_profile_read.argtypes = [vp, vp, i32]
+        L.oapl_profile_read_clocks.restype = i32
+        L.oapl_profile_read_clocks.argtypes = [vp, i32]
         _lib = L
     return _lib
 
@@ -176,8 +178,9 @@ def oapl_launch_count() -> int:
     return int(lib().oapl_launch_count())
 
 
-def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err):
-    rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), _ptr(err), _stream())
+def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err, wide=False):
+    rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), int(wide), _ptr(err),
+                               _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_debug_gemm")
 
@@ -199,6 +202,15 @@ def oapl_profile_read() -> dict:
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_profile_read")
     return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KINDS)}
+
+
+def oapl_profile_read_clocks() -> dict:
+    """{kind: SM MHz the kind's launches ran at} since the last read (0 = did not run)."""
+    mhz = (ctypes.c_float * len(KINDS))()
+    rc = lib().oapl_profile_read_clocks(mhz, len(KINDS))
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_profile_read_clocks")
+    return {k: float(mhz[i]) for i, k in enumerate(KINDS)}
 
 
 def oapl_token_logprobs_static(problem, token_logp, seq_logp, device_status=None):

@@ -14,10 +14,18 @@
 // by one SM only, without multicast), the leader CTA's UMMA thread issues for both, and
 // each CTA's TMEM receives its 128 rows of the accumulator.
 // CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM (and, in the leader, issues the
-// UMMAs), warps 2..5 are the epilogue (one TMEM lane quadrant each).  Six shared-memory
-// stages of 32 KB per CTA, two 256-column fp32 accumulators in TMEM so that the epilogue of
-// tile j overlaps the main loop of tile j+1.  bf16 tiles leave through shared memory and
-// TMA stores.
+// UMMAs), warps 2..5 are the epilogue (one TMEM lane quadrant each).
+//
+// Two tile shapes (template parameter NACC):
+//   NACC = 1  256 x 256 pair tile, six shared-memory stages of 32 KB per CTA, the two
+//             256-column fp32 accumulators in TMEM alternate so that the epilogue of tile j
+//             overlaps the main loop of tile j+1 (the vocabulary sweeps: short K = d, heavy
+//             epilogue).  bf16 tiles leave through shared memory and TMA stores.
+//   NACC = 2  256 x 512 pair tile: both accumulators belong to one tile and every A slab
+//             feeds two UMMAs, so a third less operand traffic from L2 per flop and half as
+//             many re-reads of the streamed operand from HBM; four stages of 48 KB.  The
+//             epilogue is not overlapped, which is why only the contractions with a long K
+//             (dH: K = V, dW: K = rows of the range) use it.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -33,15 +41,23 @@ constexpr int kBM = 128;      // rows of A / of the accumulator per CTA
 constexpr int kTileM = 256;   // rows per CTA pair
 constexpr int kBN = 256;      // accumulator columns (per pair and per CTA)
 constexpr int kHalfN = 128;   // columns of B each CTA loads
-constexpr int kBK = 64, kStages = 6;
+constexpr int kBK = 64;
 constexpr int kABytes = kBM * kBK * 2;     // 16 KB
 constexpr int kBBytes = kHalfN * kBK * 2;  // 16 KB
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kOutBytes = kBM * 64 * 2;  // one 128 x 64 bf16 output piece (16 KB), two of them
 constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr size_t kGemmSmemBytes =
-    size_t(kStages) * kStageBytes + 2 * kOutBytes + 1024 /*align*/ + 256 /*barriers*/;
+
+// Shared-memory plan of the two tile shapes.
+template <int NACC>
+struct TileCfg {
+  static constexpr int kStages = NACC == 2 ? 4 : 6;
+  static constexpr int kStageBytes = kABytes + NACC * kBBytes;
+  static constexpr int kOutTotal = NACC == 2 ? 0 : 2 * kOutBytes;
+  static constexpr int kTileN = NACC * kBN;  // columns of one pair tile
+  static constexpr size_t kSmemBytes =
+      size_t(kStages) * kStageBytes + kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
+};
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kErrTimeout = -8;  // OAPL_ERR_DEVICE_TIMEOUT
@@ -75,22 +91,27 @@ struct GemmParams {
   float* Cdbg;
   int M, N, K;
   int* err;  // device status word
+  // optional timing: {SM cycles, nanoseconds} of CTA 0, added up per launch (null = off)
+  unsigned long long* clk;
 };
 
 struct Tile {
   int m0, n0;    // tile origin (A's M coordinate, B's N coordinate)
   int ka0, kb0;  // K origin for the A and B tensor maps
   int nk;        // K steps of 64
+  int nh;        // 256-column accumulators in use (2 only for a wide tile that is not cut by the edge)
   int first, last, split;
 };
 
 // Tile j of this CTA pair for rows [row_begin, row_end) of the compacted row space.
 // m0 is the pair's first row; CTA `rank` of the pair owns rows m0 + 128*rank ....
-template <int MODE>
+template <int MODE, int NACC>
 __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int row_end, int j,
                                          Tile& t) {
+  constexpr int kTN = NACC * kBN;
   t.first = t.last = 1;
   t.split = 0;
+  t.nh = 1;
   const int rows = row_end - row_begin;
   const int pid = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
@@ -131,31 +152,34 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
     return true;
   } else if (MODE == MODE_DH) {
     if (rows <= 0) return false;
-    const int MB = (rows + kTileM - 1) / kTileM, NB = (p.d + kBN - 1) / kBN;
+    const int MB = (rows + kTileM - 1) / kTileM, NB = (p.d + kTN - 1) / kTN;
     const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
     t.m0 = (tix / NB) * kTileM;  // row inside the staged chunk
-    t.n0 = (tix % NB) * kBN;
+    t.n0 = (tix % NB) * kTN;
+    t.nh = (NACC == 2 && t.n0 + kBN < p.d) ? 2 : 1;
     t.ka0 = t.kb0 = 0;
     t.nk = (p.V + kBK - 1) / kBK;
     return true;
   } else if (MODE == MODE_DW) {
     if (rows <= 0) return false;
-    const int MB = (p.V + kTileM - 1) / kTileM, NB = (p.d + kBN - 1) / kBN;
+    const int MB = (p.V + kTileM - 1) / kTileM, NB = (p.d + kTN - 1) / kTN;
     const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
     t.m0 = (tix / NB) * kTileM;  // vocabulary row
-    t.n0 = (tix % NB) * kBN;
+    t.n0 = (tix % NB) * kTN;
+    t.nh = (NACC == 2 && t.n0 + kBN < p.d) ? 2 : 1;
     t.ka0 = 0;          // staged chunk rows are range-relative
     t.kb0 = row_begin;  // compacted H rows are absolute
     t.nk = (rows + kBK - 1) / kBK;
     return true;
   } else {
-    const int MB = (p.M + kTileM - 1) / kTileM, NB = (p.N + kBN - 1) / kBN;
+    const int MB = (p.M + kTileM - 1) / kTileM, NB = (p.N + kTN - 1) / kTN;
     const int tix = pid + j * npairs;
     if (tix >= MB * NB) return false;
     t.m0 = (tix / NB) * kTileM;
-    t.n0 = (tix % NB) * kBN;
+    t.n0 = (tix % NB) * kTN;
+    t.nh = (NACC == 2 && t.n0 + kBN < p.N) ? 2 : 1;
     t.ka0 = t.kb0 = 0;
     t.nk = p.K / kBK;
     return true;
@@ -187,18 +211,24 @@ __device__ __forceinline__ bool epilogue_all(bool ok) {
   return r != 0;
 }
 
-template <int MODE, int A_MN, int B_MN>
+template <int MODE, int A_MN, int B_MN, int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
+  static_assert(NACC == 1 || (MODE != MODE_LSE && MODE != MODE_GRAD && MODE != MODE_LSE_E),
+                "the vocabulary sweeps need the alternating accumulators of the 256 x 256 tile");
+  using Cfg = TileCfg<NACC>;
+  constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  uint8_t* out_smem = smem + kStages * kStageBytes;  // two 16 KB output pieces
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + 2 * kOutBytes);
-  const uint32_t bar0 = base + kStages * kStageBytes + 2 * kOutBytes;
-  // barrier slots: full[0..3], empty[4..7], tmem_full[8..9], tmem_empty[10..11]
+  uint8_t* out_smem = smem + kStages * kStageBytes;  // two 16 KB output pieces (NACC = 1 only)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + Cfg::kOutTotal);
+  const uint32_t bar0 = base + kStages * kStageBytes + Cfg::kOutTotal;
+  // barrier slots: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2].
+  // NACC = 1: accumulator b = j & 1 of tile j uses tmem_full[b] / tmem_empty[b].
+  // NACC = 2: tmem_full[0] covers both halves of a tile, tmem_empty[h] releases half h.
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
@@ -208,6 +238,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();  // 0 = leader of the pair
+  long long clk0 = 0;
+  unsigned long long ns0 = 0;
+  if (p.clk && blockIdx.x == 0 && threadIdx.x == 0) {
+    clk0 = clock64();
+    ns0 = global_timer_ns();
+  }
   int row_begin = 0, row_end = 0;
   if (MODE != MODE_DEBUG) {
     int n_live = *p.n_live_ptr;
@@ -249,30 +285,39 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       Tile t;
       bool ok = true;
-      for (int j = 0; ok && get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
+      for (int j = 0; ok && get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
         for (int kb = 0; kb < t.nk; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
-          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+          const uint32_t sa = base + s * kStageBytes;
           // the leader's barrier collects the bytes of both CTAs' loads
           const uint32_t fb = mapa_shared(full_bar(s), 0);
-          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * kStageBytes);
+          if (rank == 0) mbar_expect_tx(full_bar(s), 2 * (kABytes + t.nh * kBBytes));
           const int ka = t.ka0 + kb * kBK, kbb = t.kb0 + kb * kBK;
-          const int am = t.m0 + (int)rank * kBM, bn = t.n0 + (int)rank * kHalfN;
+          const int am = t.m0 + (int)rank * kBM;
           if (A_MN) {
 #pragma unroll
             for (int b = 0; b < kBM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, fb, am + 64 * b, ka);
           } else {
             tma_load_2d(sa, &tmA, fb, ka, am);
           }
-          if (B_MN) {
 #pragma unroll
-            for (int b = 0; b < kHalfN / 64; ++b) tma_load_2d(sb + b * 8192, &tmB, fb, bn + 64 * b, kbb);
-          } else {
-            tma_load_2d(sb, &tmB, fb, kbb, bn);
+          for (int h = 0; h < NACC; ++h) {
+            if (h < t.nh) {
+              // this CTA's 128 of the 256 columns of accumulator h
+              const uint32_t sb = sa + kABytes + h * kBBytes;
+              const int bn = t.n0 + h * kBN + (int)rank * kHalfN;
+              if (B_MN) {
+#pragma unroll
+                for (int b = 0; b < kHalfN / 64; ++b)
+                  tma_load_2d(sb + b * 8192, &tmB, fb, bn + 64 * b, kbb);
+              } else {
+                tma_load_2d(sb, &tmB, fb, kbb, bn);
+              }
+            }
           }
         }
       }
@@ -284,11 +329,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       Tile t;
       bool ok = true;
-      for (int j = 0; ok && get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
-        const int buf = j & 1;
-        if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
+      for (int j = 0; ok && get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
+        uint32_t d_tmem;
+        if (NACC == 1) {
+          const int buf = j & 1;
+          if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
+          d_tmem = tmem_base + buf * kBN;
+        } else {
+          // both halves of the previous tile must have been drained
+          if (!mbar_wait(tempty_bar(0), (j & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait(tempty_bar(1), (j & 1u) ^ 1u, abort_flag)) break;
+          d_tmem = tmem_base;
+        }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * kBN;
         for (int kb = 0; kb < t.nk; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag)) {
@@ -296,18 +349,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             break;
           }
           tc_fence_after();
-          const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+          const uint32_t sa = base + s * kStageBytes;
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
             const uint64_t da = A_MN ? smem_desc_sw128(sa + kk * 2048, 8192, 1024)
                                      : smem_desc_sw128(sa + kk * 32, 16, 1024);
-            const uint64_t db = B_MN ? smem_desc_sw128(sb + kk * 2048, 8192, 1024)
-                                     : smem_desc_sw128(sb + kk * 32, 16, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb | kk) ? 1u : 0u);
+#pragma unroll
+            for (int h = 0; h < NACC; ++h) {
+              if (h < t.nh) {
+                const uint32_t sb = sa + kABytes + h * kBBytes;
+                const uint64_t db = B_MN ? smem_desc_sw128(sb + kk * 2048, 8192, 1024)
+                                         : smem_desc_sw128(sb + kk * 32, 16, 1024);
+                umma_bf16(d_tmem + h * kBN, da, db, idesc, (kb | kk) ? 1u : 0u);
+              }
+            }
           }
           umma_commit_pair(empty_bar(s));  // both CTAs' stage reusable once these UMMAs have read it
         }
-        if (ok) umma_commit_pair(tfull_bar(buf));  // accumulator complete in both CTAs
+        // accumulator(s) complete in both CTAs
+        if (ok) umma_commit_pair(tfull_bar(NACC == 1 ? (j & 1) : 0));
       }
     }
   } else {
@@ -318,8 +378,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // running state of this thread's row across the tiles of a sweep
     float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f;
     Tile t;
-    for (int j = 0; get_tile<MODE>(p, row_begin, row_end, j, t); ++j) {
-      const int buf = j & 1;
+    for (int j = 0; get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
+      const int buf = NACC == 1 ? (j & 1) : 0;
       // MODE_LSE/GRAD/LSE_E: compacted row; DH: row inside the staged chunk; DW: vocabulary row
       const int row = t.m0 + (int)rank * kBM + r_in_tile;
       int tgt = -1;
@@ -338,7 +398,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           ref2 = p.lse[row] * kLog2e;
         }
       }
-      const bool got = mbar_wait(tfull_bar(buf), (j >> 1) & 1u, abort_flag);
+      const bool got = mbar_wait(tfull_bar(buf), (NACC == 1 ? (j >> 1) : j) & 1u, abort_flag);
       if (!epilogue_all(got)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;
@@ -404,11 +464,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       } else {
 #pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
+        for (int c = 0; c < t.nh * (kBN / 32); ++c) {
           uint32_t r[32];
           tmem_ld32(taddr + c * 32, r);
           tmem_ld_wait();
           const int col0 = t.n0 + c * 32;
+          if (NACC == 2 && c == kBN / 32) {
+            // first half drained: the next tile's UMMAs may overwrite it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(0), 0));
+          }
           if (MODE == MODE_LSE) {
             if (col0 < p.V) {
               float v[32];
@@ -463,10 +529,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               }
             }
           } else {
-            if (row < p.M) {
+            if (row < p.M && col0 < p.N) {  // N is a multiple of 8
+              float4* dst = reinterpret_cast<float4*>(p.Cdbg + (size_t)row * p.N + col0);
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (col0 + i < p.N) p.Cdbg[(size_t)row * p.N + col0 + i] = __uint_as_float(r[i]);
+              for (int q = 0; q < 8; ++q)
+                if (col0 + 4 * q < p.N)
+                  dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                       __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
             }
           }
         }
@@ -474,7 +543,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // accumulator drained: hand the TMEM buffer back to the UMMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+      if (lane == 0) {
+        if (NACC == 1) {
+          mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+        } else {
+          if (t.nh == 1) mbar_arrive_cluster(mapa_shared(tempty_bar(0), 0));
+          mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
+        }
+      }
       if (MODE == MODE_LSE || MODE == MODE_LSE_E) {
         if (t.last && valid) {
           const size_t o = (size_t)row * kMaxSplits + t.split;
@@ -504,6 +580,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (p.clk && blockIdx.x == 0 && threadIdx.x == 0) {
+    atomicAdd(p.clk, (unsigned long long)(clock64() - clk0));
+    atomicAdd(p.clk + 1, global_timer_ns() - ns0);
   }
 }
 

@@ -168,6 +168,12 @@ static cudaEvent_t g_prof_ev[kProfSlots][2];
 static int g_prof_kind[kProfSlots];
 static bool g_prof_made = false;
 
+// {SM cycles, nanoseconds} of CTA 0 of every contraction launch, summed per kind while
+// the timing is enabled; their ratio is the SM clock the kind ran at.
+constexpr int kProfKinds = 8;
+static __device__ unsigned long long g_prof_clk[kProfKinds][2];
+static unsigned long long* g_prof_clk_addr = nullptr;
+
 static int prof_begin(int kind, cudaStream_t st) {
   if (!g_prof_on || g_prof_used >= kProfSlots) return -1;
   const int s = g_prof_used++;
@@ -179,19 +185,25 @@ static void prof_end(int slot, cudaStream_t st) {
   if (slot >= 0) cudaEventRecord(g_prof_ev[slot][1], st);
 }
 
-template <int MODE, int A_MN, int B_MN>
+template <int MODE, int A_MN, int B_MN, int NACC = 1>
 static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
                        const GemmParams& gp, int grid, cudaStream_t st) {
   static bool attr_set = false;
-  auto kern = gemm_kernel<MODE, A_MN, B_MN>;
+  auto kern = gemm_kernel<MODE, A_MN, B_MN, NACC>;
+  constexpr size_t smem = TileCfg<NACC>::kSmemBytes;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kGemmSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return OAPL_ERR_CUDA;
     attr_set = true;
   }
   const int slot = prof_begin(MODE, st);
-  kern<<<grid, kGemmThreads, kGemmSmemBytes, st>>>(a, b, c, gp);
+  if (slot >= 0 && g_prof_clk_addr) {
+    GemmParams timed = gp;
+    timed.clk = g_prof_clk_addr + 2 * MODE;
+    kern<<<grid, kGemmThreads, smem, st>>>(a, b, c, timed);
+  } else {
+    kern<<<grid, kGemmThreads, smem, st>>>(a, b, c, gp);
+  }
   OAPL_LAUNCHED();
   prof_end(slot, st);
   return cudaGetLastError() == cudaSuccess ? OAPL_OK : OAPL_ERR_CUDA;
@@ -465,9 +477,9 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
     gp.row_begin = r0;
     rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DH, 0, 1>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DH, 0, 1, 2>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
-    rc = launch_gemm<MODE_DW, 1, 1>(tmGmn, tmHmn, tmGmn, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmGmn, tmHmn, tmGmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
   return OAPL_OK;
@@ -573,10 +585,10 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
     scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, alpha, lse, ztc, rg, p->d, p->V,
                                                  c.ldg, Hs, rowscale, E);
     CKL();
-    rc = launch_gemm<MODE_DW, 1, 1>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
     gp.rowscale = rowscale;
-    rc = launch_gemm<MODE_DH, 0, 1>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DH, 0, 1, 2>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
   loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, p->S, p->P, p->beta_loss,
@@ -592,8 +604,26 @@ int oapl_profile_enable(int on) {
         if (cudaEventCreate(&g_prof_ev[i][j]) != cudaSuccess) return OAPL_ERR_CUDA;
     g_prof_made = true;
   }
+  if (on) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_prof_clk) != cudaSuccess) return OAPL_ERR_CUDA;
+    g_prof_clk_addr = static_cast<unsigned long long*>(ptr);
+    if (cudaMemset(ptr, 0, sizeof(unsigned long long) * kProfKinds * 2) != cudaSuccess) return OAPL_ERR_CUDA;
+  }
   g_prof_on = on != 0;
   g_prof_used = 0;
+  return OAPL_OK;
+}
+
+int oapl_profile_read_clocks(float* sm_mhz_by_kind, int kinds) {
+  if (!sm_mhz_by_kind || kinds <= 0 || kinds > kProfKinds) return OAPL_ERR_INVALID_ARG;
+  if (!g_prof_clk_addr) return OAPL_ERR_BAD_STATE;
+  unsigned long long h[kProfKinds][2];
+  if (cudaDeviceSynchronize() != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaMemcpy(h, g_prof_clk_addr, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return OAPL_ERR_CUDA;
+  for (int k = 0; k < kinds; ++k)
+    sm_mhz_by_kind[k] = h[k][1] ? (float)((double)h[k][0] / (double)h[k][1] * 1e3) : 0.f;
+  if (cudaMemset(g_prof_clk_addr, 0, sizeof(h)) != cudaSuccess) return OAPL_ERR_CUDA;
   return OAPL_OK;
 }
 
@@ -611,7 +641,7 @@ int oapl_profile_read(float* ms_by_kind, int* launches_by_kind, int kinds) {
 }
 
 int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn, int b_mn,
-                    int* err, void* stream) {
+                    int wide, int* err, void* stream) {
   if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return OAPL_ERR_INVALID_ARG;
   if (K % 64 || M % 8 || N % 8) return OAPL_ERR_UNSUPPORTED_SHAPE;
   const int n_sm = sm_count();
@@ -630,8 +660,15 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   gp.K = K;
   gp.err = err;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int tiles = ((M + kTileM - 1) / kTileM) * ((N + kBN - 1) / kBN);
+  const int tile_n = wide ? 2 * kBN : kBN;
+  const int tiles = ((M + kTileM - 1) / kTileM) * ((N + tile_n - 1) / tile_n);
   const int grid = 2 * (tiles < n_sm / 2 ? tiles : n_sm / 2);
+  if (wide) {
+    if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0, 2>(ta, tb, ta, gp, grid, st);
+    if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1, 2>(ta, tb, ta, gp, grid, st);
+    if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0, 2>(ta, tb, ta, gp, grid, st);
+    return launch_gemm<MODE_DEBUG, 1, 1, 2>(ta, tb, ta, gp, grid, st);
+  }
   if (!a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 0, 0>(ta, tb, ta, gp, grid, st);
   if (!a_mn && b_mn) return launch_gemm<MODE_DEBUG, 0, 1>(ta, tb, ta, gp, grid, st);
   if (a_mn && !b_mn) return launch_gemm<MODE_DEBUG, 1, 0>(ta, tb, ta, gp, grid, st);

@@ -72,7 +72,7 @@ def test_argument_errors_return_before_any_device_work(L):
     assert L.oapl_token_logprobs(ctypes.byref(p), None, None, ws, n, 0, st) == -1
     assert L.oapl_value_estimate(out, out, 8, 2, -1.0, out, st) == -1
     assert L.oapl_value_estimate(None, out, 8, 2, 1.0, out, st) == -1
-    assert L.oapl_debug_gemm(out, out, out, 128, 256, 100, 0, 0, None, st) == -4
+    assert L.oapl_debug_gemm(out, out, out, 128, 256, 100, 0, 0, 0, None, st) == -4
 
 
 def test_status_strings(L):

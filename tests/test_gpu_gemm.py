@@ -9,9 +9,11 @@ from paper_2602_19362_b200 import binding as B, synth
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("wide", [False, True], ids=["256x256", "256x512"])
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1), (1, 0)])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (384, 512, 320), (200, 264, 128), (1000, 1304, 1088)])
-def test_debug_gemm(M, N, K, a_mn, b_mn):
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (384, 512, 320), (200, 264, 128), (1000, 1304, 1088),
+                                   (520, 3000, 4096)])
+def test_debug_gemm(M, N, K, a_mn, b_mn, wide):
     g = torch.Generator().manual_seed(M * 7 + N * 3 + K + a_mn * 2 + b_mn)
     A = torch.randn(M, K, generator=g).to(torch.bfloat16)
     Bm = torch.randn(N, K, generator=g).to(torch.bfloat16)     # C = A . Bm^T
@@ -20,7 +22,7 @@ def test_debug_gemm(M, N, K, a_mn, b_mn):
     B_dev = (Bm.t().contiguous() if b_mn else Bm).cuda()
     C = torch.full((M, N), float("nan"), device="cuda")
     err = torch.zeros(1, dtype=torch.int32, device="cuda")
-    B.oapl_debug_gemm(A_dev, B_dev, C, M, N, K, a_mn, b_mn, err)
+    B.oapl_debug_gemm(A_dev, B_dev, C, M, N, K, a_mn, b_mn, err, wide=wide)
     torch.cuda.synchronize()
     assert int(err.item()) == 0
     got = C.cpu().numpy().astype(np.float64)
