@@ -141,6 +141,25 @@ int oapl_loss_fwd_bwd(const oapl_problem* problem /*host*/, float* loss, float* 
                       float* delta /*may be NULL*/, float* token_logp /*may be NULL*/, void* dH, float* dW,
                       int accumulate_dW, void* ws, size_t ws_bytes, int flags, void* stream);
 
+/*
+ * Policy entropy of the trainer policy on the response tokens, the training-dynamics
+ * diagnostic of the paper's experiments (the entropy curves of OAPL against GRPO in the
+ * "Training dynamics" figure and the "sequence entropy" discussed beside it):
+ *     H_n = - sum_v p[n,v] ln p[n,v] = lse_n - sum_v p[n,v] z[n,v],   p = softmax(z).
+ * Every forward of this library (oapl_token_logprobs, oapl_loss_fwd, oapl_loss_fwd_bwd)
+ * accumulates sum_v exp(z - ref) z next to the log-sum-exp in the same pass over the
+ * logits and leaves H_n per response token in the workspace; this call only reads it back:
+ *   token_entropy [N] f32 or NULL: H_n, 0 where mask==0;
+ *   seq_entropy   [S] f32 or NULL: mean of H_n over the sequence's response tokens
+ *                                  (0 for a sequence without any);
+ *   mean_entropy  [1] f32 or NULL: mean of H_n over all response tokens of the batch.
+ * `problem`, `ws`, `ws_bytes` and `flags` are those of the forward call (OAPL_FLAG_FUSED for
+ * oapl_loss_fwd_bwd).  Without a preceding forward on `ws` the status word becomes
+ * OAPL_ERR_BAD_STATE and nothing is written.
+ */
+int oapl_entropy(const oapl_problem* problem /*host*/, float* token_entropy, float* seq_entropy,
+                 float* mean_entropy, void* ws, size_t ws_bytes, int flags, void* stream);
+
 /* Synchronises `stream` and returns the status word the device recorded in `ws`
  * since the last forward call (OAPL_OK if none). */
 int oapl_get_last_status(void* ws, void* stream);
@@ -161,7 +180,7 @@ const char* oapl_status_string(int status);
  * Who needs it: code that is not allowed to allocate device memory where it calls us --
  * a plug-in inside a framework that owns the allocator, a serving loop whose memory was
  * fixed at start-up, or a section in which the CUDA allocator must not be entered.  The
- * scratch memory lives in a fixed device array inside the library (about 4.6 MB per GPU
+ * scratch memory lives in a fixed device array inside the library (about 4.8 MB per GPU
  * that loads the library, held until the process exits), so sizes are limited:
  *     N <= 2048,  d <= 1024 (multiple of 64),  S <= 2048,  any V >= 1.
  * Larger problems return OAPL_ERR_UNSUPPORTED_SHAPE and print the limits to stderr.

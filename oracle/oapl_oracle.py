@@ -26,7 +26,8 @@ normalisation, the W=0 and V=2 closed forms, scipy's logsumexp, the beta->0 and
 beta->inf limits of Eq. 2, its binary-reward closed form and a 60-digit decimal
 evaluation of the literal formula, zero loss and zero gradient at the
 closed-form optimum, central finite differences of the loss, and the zero
-column sum of dW.  The paper prints no worked numeric example, so the numeric
+column sum of dW; for the entropy statistic the literal -sum p ln p, the uniform
+and two-token closed forms, scipy.stats.entropy and the bound 0 <= H <= ln V.  The paper prints no worked numeric example, so the numeric
 end-to-end value of a whole step is "parity unpinned" beyond those pins.
 """
 from __future__ import annotations
@@ -208,6 +209,32 @@ def token_entropy(H, W, mask):
         p = np.exp(z - l[:, None])
         ent[live] = l - (p * z).sum(axis=1)
     return ent
+
+
+def sequence_entropy(ent, mask, seq_id, S):
+    """Per-sequence mean of the token entropies over the response tokens (0 for
+    a sequence without any) and the mean over all response tokens of the batch:
+    the "sequence entropy" the paper's training-dynamics figure tracks, read as
+    the token-level entropy averaged over the response."""
+    m = np.asarray(mask).astype(bool)
+    seq_id = np.asarray(seq_id).astype(np.int64)
+    ent = np.asarray(ent, dtype=np.float64)
+    per_seq = np.zeros(S)
+    for i in range(S):
+        rows = m & (seq_id == i)
+        if rows.any():
+            per_seq[i] = ent[rows].mean()
+    mean = ent[m].mean() if m.any() else 0.0
+    return per_seq, float(mean)
+
+
+def row_entropy(h, W):
+    """Entropy of one row's next-token distribution."""
+    z = np.asarray(W, dtype=np.float64) @ np.asarray(h, dtype=np.float64)
+    M = z.max()
+    e = np.exp(z - M)
+    lse = M + np.log(e.sum())
+    return lse - (e * z).sum() / e.sum()
 
 
 # --------------------------------------------------------------------------

@@ -22,7 +22,7 @@ OAPL_FLAG_FUSED = 1
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
-           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks"]
+           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.oapl_loss_fwd_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_token_logprobs_static.restype = i32
         L.oapl_token_logprobs_static.argtypes = [pp, vp, vp, vp, vp]
+        L.oapl_entropy.restype = i32
+        L.oapl_entropy.argtypes = [pp, vp, vp, vp, vp, sz, i32, vp]
         L.oapl_profile_enable.restype = i32
         L.oapl_profile_enable.argtypes = [i32]
         L.oapl_profile_read.restype = i32
@@ -164,6 +166,13 @@ def oapl_loss_bwd(problem, dH, dW, accumulate_dW, ws, flags=0):
                              ws.numel(), flags, _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_loss_bwd")
+
+
+def oapl_entropy(problem, token_entropy, seq_entropy, mean_entropy, ws, flags=0):
+    rc = lib().oapl_entropy(ctypes.byref(problem), _ptr(token_entropy), _ptr(seq_entropy), _ptr(mean_entropy),
+                            _ptr(ws), ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_entropy")
 
 
 def oapl_get_last_status(ws) -> int:

@@ -76,6 +76,7 @@ struct GemmParams {
   float* pm;
   float* pl;
   float* pz;
+  float* ps;  // sum of exp(z - ref) * z, for the policy-entropy statistic
   // per compacted row
   const int* tgt_c;
   const int* seq_c;
@@ -376,7 +377,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int r_in_tile = quad * 32 + lane;
     const bool issuer = (threadIdx.x == 64);  // issues the TMA stores of the bf16 pieces
     // running state of this thread's row across the tiles of a sweep
-    float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f;
+    float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f, run_s = 0.f;
     Tile t;
     for (int j = 0; get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
       const int buf = NACC == 1 ? (j & 1) : 0;
@@ -389,7 +390,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         valid = row < row_end;
         tgt = valid ? p.tgt_c[row] : -1;
         if (MODE == MODE_LSE_E && valid) ref2 = p.zref[row] * kLog2e;
-        if (t.first) { run_m2 = -INFINITY; run_l = 0.f; run_z = 0.f; }
+        if (t.first) { run_m2 = -INFINITY; run_l = 0.f; run_z = 0.f; run_s = 0.f; }
       } else if (MODE == MODE_GRAD) {
         valid = row < row_end;
         if (valid) {
@@ -417,17 +418,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (valid && col0 < p.V) {
               const int ti = tgt - col0;
               if (MODE == MODE_LSE_E) {
-                float acc = 0.f;
+                // columns past V hold z = 0 (zero-filled W rows): finite, and their e is cleared
+                float acc = 0.f, accs = 0.f;
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                  float e0 = ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -ref2));
-                  float e1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -ref2));
+                  const float z0 = __uint_as_float(r[i]), z1 = __uint_as_float(r[i + 1]);
+                  float e0 = ex2_approx(fmaf(z0, kLog2e, -ref2));
+                  float e1 = ex2_approx(fmaf(z1, kLog2e, -ref2));
                   if (col0 + i >= p.V) e0 = 0.f;
                   if (col0 + i + 1 >= p.V) e1 = 0.f;
                   acc += e0 + e1;
+                  accs = fmaf(e0, z0, fmaf(e1, z1, accs));
                   w[h * 16 + (i >> 1)] = pack_bf16x2(e0, e1);
                 }
                 run_l += acc;
+                run_s += accs;
                 if (ti >= 0 && ti < 32) {
 #pragma unroll
                   for (int i = 0; i < 32; ++i)
@@ -481,18 +486,25 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
               for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
               if (col0 + 32 > p.V) {
+                // a large finite negative: its exponential is 0 and 0 * v stays 0 (no NaN)
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
-                  if (col0 + i >= p.V) v[i] = -INFINITY;
+                  if (col0 + i >= p.V) v[i] = -3.0e38f;
               }
               float cmax = v[0];
 #pragma unroll
               for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
               const float m2 = fmaxf(run_m2, cmax * kLog2e);
-              float acc = 0.f;
+              float acc = 0.f, accs = 0.f;
 #pragma unroll
-              for (int i = 0; i < 32; ++i) acc += ex2_approx(fmaf(v[i], kLog2e, -m2));
-              run_l = run_l * ex2_approx(run_m2 - m2) + acc;
+              for (int i = 0; i < 32; ++i) {
+                const float e = ex2_approx(fmaf(v[i], kLog2e, -m2));
+                acc += e;
+                accs = fmaf(e, v[i], accs);
+              }
+              const float resc = ex2_approx(run_m2 - m2);
+              run_l = run_l * resc + acc;
+              run_s = run_s * resc + accs;
               run_m2 = m2;
               const int ti = tgt - col0;
               if (ti >= 0 && ti < 32) {
@@ -557,6 +569,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (MODE == MODE_LSE) p.pm[o] = run_m2 * kLn2;  // back to natural units
           p.pl[o] = run_l;
           p.pz[o] = run_z;
+          p.ps[o] = run_s;
         }
       }
     }

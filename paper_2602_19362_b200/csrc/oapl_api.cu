@@ -24,7 +24,7 @@ constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref)
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Carve {
-  size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, pm, pl, pz, cstart,
+  size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, ent_c, pm, pl, pz, ps, cstart,
       cend, seq_D, coef, vhat, seq_logp, Hc, G, zref, alpha, ztc, rowscale, Hs, ranges, total;
   int n_pad, nblk, chunk_rows, ldg;
   int stage_rows, stage_alloc_rows, max_ranges;  // single-call path only
@@ -62,9 +62,11 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
   c->q_c = take(4 * n_pad);
   c->lp_c = take(4 * n_pad);
   c->lse = take(4 * n_pad);
+  c->ent_c = take(4 * n_pad);
   c->pm = take(4 * n_pad * kMaxSplits);
   c->pl = take(4 * n_pad * kMaxSplits);
   c->pz = take(4 * n_pad * kMaxSplits);
+  c->ps = take(4 * n_pad * kMaxSplits);
   c->cstart = take(4 * (size_t)p->S);
   c->cend = take(4 * (size_t)p->S);
   c->seq_D = take(4 * (size_t)p->S);
@@ -306,13 +308,15 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.pm = reinterpret_cast<float*>(ws + c.pm);
   gp.pl = reinterpret_cast<float*>(ws + c.pl);
   gp.pz = reinterpret_cast<float*>(ws + c.pz);
+  gp.ps = reinterpret_cast<float*>(ws + c.ps);
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
   int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
-  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.R, gp.C, (p->V + kBN - 1) / kBN, state,
-                                             live_rows, lse, lp_c, token_logp);
+  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.ps, gp.R, gp.C, (p->V + kBN - 1) / kBN,
+                                             state, live_rows, lse, lp_c,
+                                             reinterpret_cast<float*>(ws + c.ent_c), token_logp);
   CKL();
   seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp,
                                         reinterpret_cast<float*>(ws + c.seq_D), with_q ? 1 : 0, nullptr);
@@ -557,6 +561,7 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   gp.ldg = c.ldg;
   gp.pl = reinterpret_cast<float*>(w + c.pl);
   gp.pz = reinterpret_cast<float*>(w + c.pz);
+  gp.ps = reinterpret_cast<float*>(w + c.ps);
   gp.tgt_c = tgt_c;
   gp.zref = zref;
   gp.live_rows = live_rows;
@@ -574,8 +579,8 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
     gp.rowscale = nullptr;
     rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
-    merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
-                                         alpha, ztc, token_logp);
+    merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
+                                         reinterpret_cast<float*>(w + c.ent_c), alpha, ztc, token_logp, state);
     CKL();
     seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp, seq_D, 1, &rg->seq_begin);
     CKL();
@@ -594,6 +599,32 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, p->S, p->P, p->beta_loss,
                                  p->loss_scale, coef, delta, loss, state);
   CKL();
+  return OAPL_OK;
+}
+
+int oapl_entropy(const oapl_problem* p, float* token_entropy, float* seq_entropy, float* mean_entropy,
+                 void* ws, size_t ws_bytes, int flags, void* stream) {
+  int rc = check_problem(p, false);
+  if (rc != OAPL_OK) return rc;
+  if (!ws || (!token_entropy && !seq_entropy && !mean_entropy)) return OAPL_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, flags, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  DevState* state = reinterpret_cast<DevState*>(w + c.state);
+  const float* ent_c = reinterpret_cast<const float*>(w + c.ent_c);
+  if (token_entropy) CK(cudaMemsetAsync(token_entropy, 0, 4 * (size_t)p->N, st));
+  entropy_seq_kernel<<<p->S, 256, 0, st>>>(ent_c, reinterpret_cast<const int*>(w + c.cstart),
+                                           reinterpret_cast<const int*>(w + c.cend),
+                                           reinterpret_cast<const int*>(w + c.live_rows), token_entropy,
+                                           seq_entropy, state);
+  CKL();
+  if (mean_entropy) {
+    entropy_mean_kernel<<<1, 1024, 0, st>>>(ent_c, state, mean_entropy);
+    CKL();
+  }
   return OAPL_OK;
 }
 
@@ -682,15 +713,15 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
 // to allocate device memory at the point of the call: a plug-in running inside a host
 // framework that owns the allocator, a latency-critical serving loop whose memory was fixed
 // at start-up, or a region of code where the CUDA allocator must not be entered.  For them
-// the scratch of oapl_token_logprobs lives in the fixed device array below (about 4.6 MB,
+// the scratch of oapl_token_logprobs lives in the fixed device array below (about 4.8 MB,
 // resident on every GPU that loads the library until the process exits), which bounds the
 // problem size: N <= 2048 rows, d <= 1024, S <= 2048 sequences, any V.
 constexpr int kStaticMaxRows = 2048;
 constexpr int kStaticMaxD = 1024;
 constexpr int kStaticMaxSeq = 2048;
 constexpr size_t kStaticScratchBytes =
-    1024 /*state*/ + 2 * 1024 /*block counts, offsets*/ + 6 * 4 * (size_t)kStaticMaxRows /*per-row arrays*/ +
-    3 * 4 * (size_t)kStaticMaxRows * kMaxSplits /*log-sum-exp partials*/ +
+    1024 /*state*/ + 2 * 1024 /*block counts, offsets*/ + 7 * 4 * (size_t)kStaticMaxRows /*per-row arrays*/ +
+    4 * 4 * (size_t)kStaticMaxRows * kMaxSplits /*log-sum-exp partials*/ +
     3 * 4 * (size_t)kStaticMaxSeq /*per-sequence arrays*/ +
     2 * (size_t)kStaticMaxRows * kStaticMaxD /*compacted H*/ + 16 * 1024 /*alignment slack*/;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -751,9 +782,11 @@ int oapl_token_logprobs_static(const oapl_problem* p, float* token_logp, float* 
   c.q_c = take(4 * n_pad);
   c.lp_c = take(4 * n_pad);
   c.lse = take(4 * n_pad);
+  c.ent_c = take(4 * n_pad);
   c.pm = take(4 * n_pad * kMaxSplits);
   c.pl = take(4 * n_pad * kMaxSplits);
   c.pz = take(4 * n_pad * kMaxSplits);
+  c.ps = take(4 * n_pad * kMaxSplits);
   c.cstart = take(4 * (size_t)p->S);
   c.cend = take(4 * (size_t)p->S);
   c.seq_D = take(4 * (size_t)p->S);

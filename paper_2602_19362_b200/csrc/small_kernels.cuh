@@ -17,8 +17,9 @@ struct DevState {
   int n_live;    // live rows counted by the last forward
   int status;    // first device-detected error (0 = none)
   int fwd_tag;   // set by the forward, checked by the backward
-  int reserved;
+  int ent_tag;   // set once the forward has left per-row entropies in the workspace
 };
+constexpr int kEntTag = 0x0E27;
 
 __device__ __forceinline__ void set_error(int* status, int code) { atomicCAS(status, 0, code); }
 
@@ -163,26 +164,31 @@ __global__ void zero_dead_rows_kernel(const uint8_t* __restrict__ mask, long lon
 
 // ---- merge the per-split (max, sum-exp, target-logit) partials ----------------------
 // Row i has sweep_splits_of_block(...) partials in slots [i*kMaxSplits, ...).
+// Also the row's policy entropy -sum_v p ln p = lse - (sum_v e^{z-M} z) / (sum_v e^{z-M}).
 __global__ void merge_lse_kernel(const float* __restrict__ pm, const float* __restrict__ pl,
-                                 const float* __restrict__ pz, int R, int C, int vtiles,
-                                 const DevState* st, const int* __restrict__ live_rows,
+                                 const float* __restrict__ pz, const float* __restrict__ ps, int R, int C,
+                                 int vtiles, DevState* st, const int* __restrict__ live_rows,
                                  float* __restrict__ lse, float* __restrict__ lp_c,
-                                 float* __restrict__ token_logp) {
+                                 float* __restrict__ ent_c, float* __restrict__ token_logp) {
   const int n_live = st->n_live;
+  if (blockIdx.x == 0 && threadIdx.x == 0) st->ent_tag = kEntTag;
   const int nrb = (n_live + kSweepRows - 1) / kSweepRows;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_live; i += gridDim.x * blockDim.x) {
     const int ns = sweep_splits_of_block(i / kSweepRows, nrb, R, C, vtiles);
     const size_t o = (size_t)i * kMaxSplits;
     float M = -INFINITY;
     for (int s = 0; s < ns; ++s) M = fmaxf(M, pm[o + s]);
-    float L = 0.f, z = 0.f;
+    float L = 0.f, z = 0.f, sz = 0.f;
     for (int s = 0; s < ns; ++s) {
-      L += pl[o + s] * expf(pm[o + s] - M);
+      const float w = expf(pm[o + s] - M);
+      L += pl[o + s] * w;
+      sz += ps[o + s] * w;
       z += pz[o + s];
     }
     const float l = M + logf(L);
     lse[i] = l;
     lp_c[i] = z - l;
+    ent_c[i] = l - sz / L;
     if (token_logp) token_logp[live_rows[i]] = z - l;
   }
 }
@@ -373,23 +379,27 @@ __global__ void plan_ranges_kernel(const int* __restrict__ cstart, const int* __
 
 // lse = zref + ln(sum_v e), token log-prob, and alpha = exp(zref - lse) = 1 / sum_v e.
 __global__ void merge_e_kernel(const float* __restrict__ pl, const float* __restrict__ pz,
-                               const float* __restrict__ zref, const RangeRec* __restrict__ range, int R,
-                               int C, int vtiles, const int* __restrict__ live_rows,
-                               float* __restrict__ lse, float* __restrict__ lp_c,
+                               const float* __restrict__ ps, const float* __restrict__ zref,
+                               const RangeRec* __restrict__ range, int R, int C, int vtiles,
+                               const int* __restrict__ live_rows, float* __restrict__ lse,
+                               float* __restrict__ lp_c, float* __restrict__ ent_c,
                                float* __restrict__ alpha, float* __restrict__ ztc,
-                               float* __restrict__ token_logp) {
+                               float* __restrict__ token_logp, DevState* st) {
   const int rb = range->row_begin, re = range->row_end;
+  if (blockIdx.x == 0 && threadIdx.x == 0) st->ent_tag = kEntTag;
   const int nrb = (re - rb + kSweepRows - 1) / kSweepRows;
   for (int i = rb + blockIdx.x * blockDim.x + threadIdx.x; i < re; i += gridDim.x * blockDim.x) {
     const int ns = sweep_splits_of_block((i - rb) / kSweepRows, nrb, R, C, vtiles);
     const size_t o = (size_t)i * kMaxSplits;
-    float L = 0.f, z = 0.f;
+    float L = 0.f, z = 0.f, sz = 0.f;
     for (int s = 0; s < ns; ++s) {
       L += pl[o + s];
+      sz += ps[o + s];
       z += pz[o + s];
     }
     const float l = zref[i] + logf(L);
     lse[i] = l;
+    ent_c[i] = l - sz / L;
     ztc[i] = z;
     alpha[i] = 1.f / L;
     lp_c[i] = z - l;
@@ -453,6 +463,58 @@ __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const i
     } else {
       for (int k = lane; k < vec; k += 32) dst[k] = make_uint4(0, 0, 0, 0);
     }
+  }
+}
+
+// =====================================================================================
+// Policy-entropy statistic read back from what a forward left in the workspace.
+// =====================================================================================
+// One CTA per sequence: mean of the per-row entropies over the sequence's response tokens
+// (0 for a sequence without any), and the scatter of the per-row values to their rows.
+__global__ void entropy_seq_kernel(const float* __restrict__ ent_c, const int* __restrict__ cstart,
+                                   const int* __restrict__ cend, const int* __restrict__ live_rows,
+                                   float* __restrict__ token_entropy, float* __restrict__ seq_entropy,
+                                   DevState* st) {
+  __shared__ double sh[8];
+  if (st->ent_tag != kEntTag) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) set_error(&st->status, -10);
+    return;
+  }
+  const int s = blockIdx.x;
+  const int b = cstart[s], e = cend[s];
+  double acc = 0.0;
+  for (int i = b + threadIdx.x; i < e; i += blockDim.x) {
+    const float h = ent_c[i];
+    acc += h;
+    if (token_entropy) token_entropy[live_rows[i]] = h;
+  }
+  acc = warp_sum_d(acc);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) sh[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0 && seq_entropy) {
+    double t = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
+    seq_entropy[s] = e > b ? (float)(t / (double)(e - b)) : 0.f;
+  }
+}
+
+// Mean over all response tokens of the batch (one CTA, fixed order; 0 when none is live).
+__global__ void entropy_mean_kernel(const float* __restrict__ ent_c, const DevState* st,
+                                    float* __restrict__ mean_entropy) {
+  __shared__ double sh[32];
+  if (st->ent_tag != kEntTag) return;
+  const int n_live = st->n_live;
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n_live; i += blockDim.x) acc += ent_c[i];
+  acc = warp_sum_d(acc);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) sh[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
+    *mean_entropy = n_live > 0 ? (float)(t / (double)n_live) : 0.f;
   }
 }
 

@@ -311,3 +311,33 @@ def test_entropy_definition():
         pr = np.exp(z) / np.exp(z).sum()
         assert ent[n] == pytest.approx(-(pr * np.log(pr)).sum(), abs=1e-12)
     assert orc.token_entropy(H, np.zeros_like(W), mask)[0] == pytest.approx(math.log(W.shape[0]))
+
+
+def test_entropy_closed_forms_bounds_and_scipy():
+    import scipy.stats
+    r = np.random.default_rng(7)
+    # two-token vocabulary: binary entropy of the logistic of the logit gap
+    H = r.normal(size=(6, 4))
+    W = r.normal(size=(2, 4))
+    ent = orc.token_entropy(H, W, np.ones(6, dtype=np.uint8))
+    gap = H @ (W[0] - W[1])
+    q = 1.0 / (1.0 + np.exp(-gap))
+    assert np.allclose(ent, -(q * np.log(q) + (1 - q) * np.log1p(-q)), atol=1e-12)
+    # a different library routine on explicit probabilities; bounds; one-hot limit
+    H, W, _, mask, seq_id = _tiny(N=9, d=6, V=13, S=3, seed=3)
+    ent = orc.token_entropy(H, W, mask)
+    p = scipy.special.softmax(H @ W.T, axis=1)
+    want = scipy.stats.entropy(p, axis=1)
+    assert np.allclose(ent[mask == 1], want[mask == 1], atol=1e-12)
+    assert np.all(ent >= 0) and np.all(ent <= math.log(13) + 1e-12)
+    assert orc.token_entropy(50.0 * H, W, mask).max() < ent.max()          # sharper logits, lower entropy
+    assert orc.row_entropy(H[0], W) == pytest.approx(ent[0], abs=1e-12)
+    # per-sequence and batch means by explicit loops
+    per_seq, mean = orc.sequence_entropy(ent, mask, seq_id, 3)
+    tot, cnt = 0.0, 0
+    for i in range(3):
+        vals = [ent[n] for n in range(9) if mask[n] and seq_id[n] == i]
+        assert per_seq[i] == pytest.approx(sum(vals) / len(vals) if vals else 0.0, abs=1e-14)
+        tot, cnt = tot + sum(vals), cnt + len(vals)
+    assert mean == pytest.approx(tot / cnt, abs=1e-14)
+    assert orc.sequence_entropy(ent, np.zeros(9, dtype=np.uint8), seq_id, 3)[1] == 0.0
