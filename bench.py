@@ -3,11 +3,12 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl reference]
 
-A step is one oapl_loss_fwd + oapl_loss_bwd over one synthetic batch shaped like the
-paper's 7B-scale trainer step (d=3584, V=152064, 16 prompts x 8 rollouts, response
-lengths U[512,4096], padded layout).  The metric is response tokens per second; the
-roofline object credits 6*N*d*V flops per step against the measured dense-bf16 peak.
-Rank 0 prints one JSON line.
+A step is one oapl_loss_fwd_bwd call (Eq. 3 forward and gradient; `--path two-calls` times
+oapl_loss_fwd + oapl_loss_bwd instead) over one synthetic batch shaped like the paper's
+7B-scale trainer step (d=3584, V=152064, 16 prompts x 8 rollouts, response lengths
+U[512,4096], padded layout).  The metric is response tokens per second; the roofline
+object credits 6*N*d*V flops per step against the measured dense-bf16 peak.  Rank 0
+prints one JSON line.
 """
 from __future__ import annotations
 
@@ -214,8 +215,22 @@ def run_cuda(args) -> None:
     dH = torch.empty(N, d, dtype=torch.bfloat16, device=dev)
     dW = torch.empty(V, d, dtype=torch.float32, device=dev)
 
+    grpo = args.objective == "grpo"
+    if grpo:
+        # the paper's baseline on the same pipeline: pi_old = the engine's log-probs plus noise,
+        # group-normalised advantages, clip ratio 0.2
+        if not fused:
+            raise SystemExit("--objective grpo runs on the single-call path only")
+        gen = torch.Generator(device=dev).manual_seed(args.seed + 1000 + rank)
+        logp_old = batch["logp_inf"] + 0.1 * torch.randn(N, device=dev, generator=gen)
+        adv = torch.zeros(S, device=dev)
+        B.oapl_group_advantage(batch["reward"], batch["group_id"], P, 1e-6, adv)
+        clip_frac = torch.zeros(1, device=dev)
+
     def step():
-        if fused:
+        if grpo:
+            B.oapl_grpo_loss_fwd_bwd(prob, logp_old, adv, 0.2, loss, seq_logp, None, clip_frac, dH, dW, False, ws)
+        elif fused:
             B.oapl_loss_fwd_bwd(prob, loss, seq_logp, vhat, delta, None, dH, dW, False, ws)
         else:
             B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
@@ -329,7 +344,9 @@ def run_cuda(args) -> None:
                                    f"lengths {wl.length}, padded_to={wl.padded_to}, beta={batch['beta_v']}",
                        "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts",
                        "l2": "inputs larger than L2 (H, W, g chunk each > 126 MB); no flush needed",
-                       "api": "oapl_loss_fwd_bwd" if fused else "oapl_loss_fwd + oapl_loss_bwd",
+                       "api": ("oapl_grpo_loss_fwd_bwd" if grpo else "oapl_loss_fwd_bwd") if fused
+                              else "oapl_loss_fwd + oapl_loss_bwd",
+                       "objective": args.objective,
                        "step_ms": step_ms, "loss": loss_val},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": cpu_base}
@@ -352,6 +369,8 @@ def main() -> None:
     ap.add_argument("--samples", type=int, default=0, help="override rollouts per prompt (profiling)")
     ap.add_argument("--path", default="single-call", choices=["single-call", "two-calls"],
                     help="oapl_loss_fwd_bwd (no recompute) or oapl_loss_fwd + oapl_loss_bwd")
+    ap.add_argument("--objective", default="oapl", choices=["oapl", "grpo"],
+                    help="Eq. 3 (default, the headline metric) or the paper's GRPO baseline objective")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -142,6 +142,40 @@ int oapl_loss_fwd_bwd(const oapl_problem* problem /*host*/, float* loss, float* 
                       int accumulate_dW, void* ws, size_t ws_bytes, int flags, void* stream);
 
 /*
+ * The paper's baseline objective on the same LM-head pass: GRPO reweighted by token-level
+ * importance ratios (the display in the Background section),
+ *     J = 1/G sum_{y in group} 1/|y| sum_t  w_t * min( r_t A, clip(r_t, 1-eps, 1+eps) A ),
+ *     w_t = pi_old(y_t|.) / pi_vllm(y_t|.)   (data: no gradient),
+ *     r_t = pi(y_t|.) / pi_old(y_t|.),       A = the rollout's normalised advantage.
+ *
+ * oapl_group_advantage: A_i = (r_i - mean_p) / (std_p + eps) over the members of the
+ * rollout's group p (population standard deviation; the paper only says "normalized
+ * advantage").  reward [S], group_id [S], advantage [S]; a group without members writes
+ * nothing.  eps >= 0.
+ *
+ * oapl_grpo_loss_fwd_bwd: loss = -loss_scale * sum_i 1/|y_i| sum_t w_t * min(...) (minimised),
+ * and its gradient: per response token c_t = dloss/dlp_t = -loss_scale/|y_i| * w_t * A_i * r_t
+ * where the unclipped branch is the minimum and 0 where the clipped (constant) branch is;
+ * g[n,v] = c_n * ([v == target_n] - p[n,v]),  dH = g . W,  dW = g^T . H.  It runs on the
+ * staged pipeline of oapl_loss_fwd_bwd (no logits tensor, no recompute) with per-token instead
+ * of per-sequence coefficients.
+ *   problem:    H, W, targets, mask, seq_id, logp_inf (= ln pi_vllm per token), loss_scale and
+ *               the sizes are read; group_id, reward and the betas are not.
+ *   logp_old    [N] f32: ln pi_old per token, read where mask==1.
+ *   advantage   [S] f32.     clip_eps >= 0 (the paper's clip ratio 0.2).
+ *   loss [1]; seq_logp [S] or NULL; token_logp [N] or NULL; clip_frac [1] or NULL: the fraction
+ *   of response tokens on the clipped branch; dH [N,d] bf16; dW [V,d] f32 (overwritten, or
+ *   added to when accumulate_dW != 0).
+ *   ws: oapl_workspace_bytes(problem, OAPL_FLAG_FUSED) bytes; same limits as oapl_loss_fwd_bwd.
+ */
+int oapl_group_advantage(const float* reward, const int32_t* group_id, int32_t S, int32_t P, float eps,
+                         float* advantage, void* stream);
+int oapl_grpo_loss_fwd_bwd(const oapl_problem* problem /*host*/, const float* logp_old,
+                           const float* advantage, float clip_eps, float* loss, float* seq_logp,
+                           float* token_logp, float* clip_frac, void* dH, float* dW, int accumulate_dW,
+                           void* ws, size_t ws_bytes, int flags, void* stream);
+
+/*
  * Policy entropy of the trainer policy on the response tokens, the training-dynamics
  * diagnostic of the paper's experiments (the entropy curves of OAPL against GRPO in the
  * "Training dynamics" figure and the "sequence entropy" discussed beside it):

@@ -196,6 +196,78 @@ def loss_bwd(H, W, targets, mask, seq_id, coef):
     return dH, dW
 
 
+# --------------------------------------------------------------------------
+# the paper's baseline: GRPO with token-level importance weights
+# (the display in the Background section)
+# --------------------------------------------------------------------------
+def group_advantage(reward, group_id, P, eps):
+    """Normalised advantage A_i = (r_i - mean_p) / (std_p + eps) over the
+    members of the rollout's group (population standard deviation)."""
+    r = np.asarray(reward, dtype=np.float64)
+    g = np.asarray(group_id).astype(np.int64)
+    adv = np.zeros_like(r)
+    for p in range(P):
+        sel = g == p
+        if sel.any():
+            adv[sel] = (r[sel] - r[sel].mean()) / (r[sel].std() + eps)
+    return adv
+
+
+def grpo_from_logprobs(lp, logp_old, logp_inf, mask, seq_id, adv, S, clip_eps, loss_scale):
+    """Loss and per-token coefficients of the importance-weighted GRPO objective.
+
+    Per response token t of rollout i, with r_t = exp(lp_t - lp_old_t) and the
+    importance ratio w_t = exp(lp_old_t - lp_inf_t) (data):
+        term_t = w_t * min(r_t A_i, clip(r_t, 1 - eps, 1 + eps) A_i)
+        loss   = -loss_scale * sum_i (1/|y_i|) sum_t term_t
+        c_t    = dloss/dlp_t = -loss_scale/|y_i| * w_t * A_i * r_t on the unclipped
+                 branch, 0 on the clipped one (a constant).
+    """
+    m = np.asarray(mask).astype(bool)
+    sid = np.asarray(seq_id).astype(np.int64)
+    lp = np.asarray(lp, dtype=np.float64)
+    N = lp.shape[0]
+    T = np.zeros(S)
+    np.add.at(T, sid, m.astype(np.float64))
+    coef = np.zeros(N)
+    clipped = np.zeros(N, dtype=bool)
+    ratio = np.ones(N)
+    loss = 0.0
+    for n in np.flatnonzero(m):
+        i = sid[n]
+        A = float(adv[i])
+        r = np.exp(lp[n] - float(logp_old[n]))
+        w = np.exp(float(logp_old[n]) - float(logp_inf[n]))
+        rc = min(max(r, 1.0 - clip_eps), 1.0 + clip_eps)
+        un, cl = r * A, rc * A
+        ratio[n] = r
+        if un <= cl:
+            term = un
+            coef[n] = -loss_scale / T[i] * w * A * r
+        else:
+            term = cl
+            clipped[n] = True
+        loss += -loss_scale / T[i] * w * term
+    n_live = int(m.sum())
+    return dict(loss=loss, coef=coef, clipped=clipped, ratio=ratio,
+                clip_frac=(clipped.sum() / n_live if n_live else 0.0), T=T)
+
+
+def grpo_fwd(H, W, targets, mask, seq_id, logp_old, logp_inf, adv, S, clip_eps, loss_scale):
+    lp, lse = token_logprobs(H, W, targets, mask)
+    out = grpo_from_logprobs(lp, logp_old, logp_inf, mask, seq_id, adv, S, clip_eps, loss_scale)
+    s, _, _ = sequence_sums(lp, np.zeros_like(lp), mask, seq_id, S)
+    out.update(token_logp=lp, lse=lse, seq_logp=s)
+    return out
+
+
+def token_coef_bwd(H, W, targets, mask, coef_tok):
+    """dH, dW for a per-token coefficient: g[n, v] = c_n ([v == y_n] - p[n, v])."""
+    H = np.asarray(H, dtype=np.float64)
+    n = H.shape[0]
+    return loss_bwd(H, W, targets, mask, np.arange(n), coef_tok)
+
+
 def token_entropy(H, W, mask):
     """Per-row policy entropy -sum_v p ln p (the diagnostic tracked in the
     paper's entropy figure); 0 on masked rows."""

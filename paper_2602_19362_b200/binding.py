@@ -22,7 +22,8 @@ OAPL_FLAG_FUSED = 1
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
-           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy"]
+           "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy", "oapl_group_advantage",
+           "oapl_grpo_loss_fwd_bwd"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.oapl_loss_fwd_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_token_logprobs_static.restype = i32
         L.oapl_token_logprobs_static.argtypes = [pp, vp, vp, vp, vp]
+        L.oapl_group_advantage.restype = i32
+        L.oapl_group_advantage.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, f32, vp, vp]
+        L.oapl_grpo_loss_fwd_bwd.restype = i32
+        L.oapl_grpo_loss_fwd_bwd.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_entropy.restype = i32
         L.oapl_entropy.argtypes = [pp, vp, vp, vp, vp, sz, i32, vp]
         L.oapl_profile_enable.restype = i32
@@ -166,6 +171,22 @@ def oapl_loss_bwd(problem, dH, dW, accumulate_dW, ws, flags=0):
                              ws.numel(), flags, _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_loss_bwd")
+
+
+def oapl_group_advantage(reward, group_id, P, eps, advantage):
+    rc = lib().oapl_group_advantage(_ptr(reward), _ptr(group_id), reward.numel(), P, eps, _ptr(advantage),
+                                    _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_group_advantage")
+
+
+def oapl_grpo_loss_fwd_bwd(problem, logp_old, advantage, clip_eps, loss, seq_logp, token_logp, clip_frac, dH, dW,
+                           accumulate_dW, ws, flags=0):
+    rc = lib().oapl_grpo_loss_fwd_bwd(ctypes.byref(problem), _ptr(logp_old), _ptr(advantage), clip_eps,
+                                      _ptr(loss), _ptr(seq_logp), _ptr(token_logp), _ptr(clip_frac), _ptr(dH),
+                                      _ptr(dW), int(accumulate_dW), _ptr(ws), ws.numel(), flags, _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_grpo_loss_fwd_bwd")
 
 
 def oapl_entropy(problem, token_entropy, seq_entropy, mean_entropy, ws, flags=0):

@@ -25,7 +25,8 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 struct Carve {
   size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, ent_c, pm, pl, pz, ps, cstart,
-      cend, seq_D, coef, vhat, seq_logp, Hc, G, zref, alpha, ztc, rowscale, Hs, ranges, total;
+      cend, seq_D, coef, vhat, seq_logp, Hc, G, zref, alpha, ztc, rowscale, Hs, ranges, coef_row, qo_c,
+      seq_obj, seq_clip, total;
   int n_pad, nblk, chunk_rows, ldg;
   int stage_rows, stage_alloc_rows, max_ranges;  // single-call path only
 };
@@ -90,9 +91,14 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
     c->rowscale = take(4 * n_pad);
     c->Hs = take(2 * (n_pad + 256) * (size_t)p->d);
     c->ranges = take(sizeof(RangeRec) * (size_t)c->max_ranges);
+    c->coef_row = take(4 * n_pad);
+    c->qo_c = take(4 * n_pad);
+    c->seq_obj = take(4 * (size_t)p->S);
+    c->seq_clip = take(4 * (size_t)p->S);
   } else {
     c->G = take(2 * (size_t)chunk * (size_t)c->ldg);
     c->zref = c->alpha = c->ztc = c->rowscale = c->Hs = c->ranges = 0;
+    c->coef_row = c->qo_c = c->seq_obj = c->seq_clip = 0;
   }
   c->total = off;
   return true;
@@ -324,6 +330,141 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   return OAPL_OK;
 }
 
+// What the staged single-call pipeline optimises: Eq. 3 (per-sequence coefficients) or
+// the GRPO display of the Background section (per-token coefficients).
+struct Objective {
+  bool grpo;
+  float* vhat;            // OAPL
+  float* delta;           // OAPL, may be null
+  const float* logp_old;  // GRPO [N]
+  const float* adv;       // GRPO [S]
+  float clip_eps;         // GRPO
+  float* clip_frac;       // GRPO, may be null
+};
+
+static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* loss, float* seq_logp,
+                          float* token_logp, void* dH, float* dW, int accumulate_dW, uint8_t* w,
+                          const Carve& c, cudaStream_t st) {
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  int rc = prologue(p, c, w, token_logp, true, st);
+  if (rc != OAPL_OK) return rc;
+  DevState* state = reinterpret_cast<DevState*>(w + c.state);
+  int* live_rows = reinterpret_cast<int*>(w + c.live_rows);
+  int* tgt_c = reinterpret_cast<int*>(w + c.tgt_c);
+  int* seq_c = reinterpret_cast<int*>(w + c.seq_c);
+  float* q_c = reinterpret_cast<float*>(w + c.q_c);
+  float* lp_c = reinterpret_cast<float*>(w + c.lp_c);
+  float* lse = reinterpret_cast<float*>(w + c.lse);
+  int* cstart = reinterpret_cast<int*>(w + c.cstart);
+  int* cend = reinterpret_cast<int*>(w + c.cend);
+  float* seq_D = reinterpret_cast<float*>(w + c.seq_D);
+  float* coef = reinterpret_cast<float*>(w + c.coef);
+  float* coef_row = reinterpret_cast<float*>(w + c.coef_row);
+  float* qo_c = reinterpret_cast<float*>(w + c.qo_c);
+  float* seq_obj = reinterpret_cast<float*>(w + c.seq_obj);
+  int* seq_clip = reinterpret_cast<int*>(w + c.seq_clip);
+  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(w + c.Hc);
+  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(w + c.G);
+  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(w + c.Hs);
+  float* zref = reinterpret_cast<float*>(w + c.zref);
+  float* alpha = reinterpret_cast<float*>(w + c.alpha);
+  float* ztc = reinterpret_cast<float*>(w + c.ztc);
+  float* rowscale = reinterpret_cast<float*>(w + c.rowscale);
+  RangeRec* ranges = reinterpret_cast<RangeRec*>(w + c.ranges);
+  const int vtiles = (p->V + kBN - 1) / kBN;
+
+  CK(cudaMemsetAsync(seq_D, 0, 4 * (size_t)p->S, st));
+  if (seq_logp) CK(cudaMemsetAsync(seq_logp, 0, 4 * (size_t)p->S, st));
+  if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
+  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH),
+                                                  nullptr);
+  CKL();
+  if (ob.grpo) {
+    CK(cudaMemsetAsync(seq_obj, 0, 4 * (size_t)p->S, st));
+    CK(cudaMemsetAsync(seq_clip, 0, 4 * (size_t)p->S, st));
+    gather_f32_kernel<<<n_sm * 4, 256, 0, st>>>(ob.logp_old, live_rows, state, qo_c);
+    CKL();
+  } else {
+    value_estimate_kernel<<<(p->P + 7) / 8, 256, 0, st>>>(p->reward, p->group_id, p->S, p->P, p->beta_v,
+                                                          ob.vhat, &state->status);
+    CKL();
+  }
+  ztgt_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, reinterpret_cast<const __nv_bfloat16*>(p->W), tgt_c, state,
+                                        p->d, p->V, zref);
+  CKL();
+  plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, c.max_ranges, ranges, state);
+  CKL();
+
+  CUtensorMap tmH, tmW, tmEk, tmWmn, tmEmn, tmHsmn;
+  const uint64_t ldg = (uint64_t)c.ldg;
+  bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
+            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
+            make_map(&tmEk, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 128) &&
+            make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
+            make_map(&tmEmn, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 64) &&
+            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 256, (uint64_t)p->d, (uint64_t)p->d, 64);
+  if (!ok) return OAPL_ERR_CUDA;
+
+  GemmParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.n_live_ptr = &state->n_live;
+  gp.d = p->d;
+  gp.V = p->V;
+  gp.ldg = c.ldg;
+  gp.pl = reinterpret_cast<float*>(w + c.pl);
+  gp.pz = reinterpret_cast<float*>(w + c.pz);
+  gp.ps = reinterpret_cast<float*>(w + c.ps);
+  gp.tgt_c = tgt_c;
+  gp.zref = zref;
+  gp.live_rows = live_rows;
+  gp.dH = static_cast<__nv_bfloat16*>(dH);
+  gp.dW = dW;
+  gp.accumulate = 1;
+  gp.err = &state->status;
+  pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
+
+  // The ranges live on the device; the host enqueues the largest number of ranges the
+  // packing can produce and launches past the last range find no work.
+  for (int k = 0; k < c.max_ranges; ++k) {
+    const RangeRec* rg = ranges + k;
+    gp.range_ptr = &rg->row_begin;
+    gp.rowscale = nullptr;
+    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
+    if (rc != OAPL_OK) return rc;
+    merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
+                                         reinterpret_cast<float*>(w + c.ent_c), alpha, ztc, token_logp, state);
+    CKL();
+    seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp, seq_D, 1, &rg->seq_begin);
+    CKL();
+    if (ob.grpo) {
+      grpo_coef_kernel<<<p->S, 256, 0, st>>>(lp_c, qo_c, q_c, cstart, cend, ob.adv, &rg->seq_begin,
+                                             ob.clip_eps, p->loss_scale, coef_row, seq_obj, seq_clip);
+      CKL();
+    } else {
+      coef_range_kernel<<<(p->S + 255) / 256, 256, 0, st>>>(p->reward, p->group_id, ob.vhat, seq_D, rg, p->P,
+                                                            p->beta_loss, p->loss_scale, coef);
+      CKL();
+    }
+    scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, ob.grpo ? coef_row : nullptr, alpha,
+                                                 lse, ztc, rg, p->d, p->V, c.ldg, Hs, rowscale, E);
+    CKL();
+    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
+    if (rc != OAPL_OK) return rc;
+    gp.rowscale = rowscale;
+    rc = launch_gemm<MODE_DH, 0, 1, 2>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
+    if (rc != OAPL_OK) return rc;
+  }
+  if (ob.grpo) {
+    grpo_loss_kernel<<<1, 256, 0, st>>>(seq_obj, seq_clip, p->S, p->loss_scale, loss, ob.clip_frac, state);
+  } else {
+    loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, ob.vhat, seq_D, p->S, p->P, p->beta_loss,
+                                   p->loss_scale, coef, ob.delta, loss, state);
+  }
+  CKL();
+  return OAPL_OK;
+}
+
 }  // namespace oapl
 
 using namespace oapl;
@@ -500,106 +641,47 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   Carve c;
   if (!carve(p, flags | OAPL_FLAG_FUSED, &c)) return OAPL_ERR_INVALID_ARG;
   if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
-  const int n_sm = sm_count();
-  if (n_sm <= 0) return OAPL_ERR_CUDA;
-  uint8_t* w = static_cast<uint8_t*>(ws);
+  Objective ob;
+  memset(&ob, 0, sizeof(ob));
+  ob.grpo = false;
+  ob.vhat = vhat;
+  ob.delta = delta;
+  return staged_fwd_bwd(p, ob, loss, seq_logp, token_logp, dH, dW, accumulate_dW, static_cast<uint8_t*>(ws), c,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int oapl_group_advantage(const float* reward, const int32_t* group_id, int32_t S, int32_t P, float eps,
+                         float* advantage, void* stream) {
+  if (!reward || !group_id || !advantage || S <= 0 || P <= 0) return OAPL_ERR_INVALID_ARG;
+  if (!(eps >= 0.f) || !std::isfinite(eps)) return OAPL_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-
-  rc = prologue(p, c, w, token_logp, true, st);
-  if (rc != OAPL_OK) return rc;
-  DevState* state = reinterpret_cast<DevState*>(w + c.state);
-  int* live_rows = reinterpret_cast<int*>(w + c.live_rows);
-  int* tgt_c = reinterpret_cast<int*>(w + c.tgt_c);
-  int* seq_c = reinterpret_cast<int*>(w + c.seq_c);
-  float* q_c = reinterpret_cast<float*>(w + c.q_c);
-  float* lp_c = reinterpret_cast<float*>(w + c.lp_c);
-  float* lse = reinterpret_cast<float*>(w + c.lse);
-  int* cstart = reinterpret_cast<int*>(w + c.cstart);
-  int* cend = reinterpret_cast<int*>(w + c.cend);
-  float* seq_D = reinterpret_cast<float*>(w + c.seq_D);
-  float* coef = reinterpret_cast<float*>(w + c.coef);
-  __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(w + c.Hc);
-  __nv_bfloat16* E = reinterpret_cast<__nv_bfloat16*>(w + c.G);
-  __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(w + c.Hs);
-  float* zref = reinterpret_cast<float*>(w + c.zref);
-  float* alpha = reinterpret_cast<float*>(w + c.alpha);
-  float* ztc = reinterpret_cast<float*>(w + c.ztc);
-  float* rowscale = reinterpret_cast<float*>(w + c.rowscale);
-  RangeRec* ranges = reinterpret_cast<RangeRec*>(w + c.ranges);
-  const int vtiles = (p->V + kBN - 1) / kBN;
-
-  CK(cudaMemsetAsync(seq_D, 0, 4 * (size_t)p->S, st));
-  CK(cudaMemsetAsync(seq_logp, 0, 4 * (size_t)p->S, st));
-  if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
-  zero_dead_rows_kernel<<<n_sm * 8, 256, 0, st>>>(p->mask, p->N, p->d, static_cast<__nv_bfloat16*>(dH),
-                                                  nullptr);
-  CKL();
-  value_estimate_kernel<<<(p->P + 7) / 8, 256, 0, st>>>(p->reward, p->group_id, p->S, p->P, p->beta_v,
-                                                        vhat, &state->status);
-  CKL();
-  ztgt_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, reinterpret_cast<const __nv_bfloat16*>(p->W), tgt_c, state,
-                                        p->d, p->V, zref);
-  CKL();
-  plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, c.max_ranges, ranges, state);
-  CKL();
-
-  CUtensorMap tmH, tmW, tmEk, tmWmn, tmEmn, tmHsmn;
-  const uint64_t ldg = (uint64_t)c.ldg;
-  bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
-            make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
-            make_map(&tmEk, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 128) &&
-            make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
-            make_map(&tmEmn, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 64) &&
-            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 256, (uint64_t)p->d, (uint64_t)p->d, 64);
-  if (!ok) return OAPL_ERR_CUDA;
-
-  GemmParams gp;
-  memset(&gp, 0, sizeof(gp));
-  gp.n_live_ptr = &state->n_live;
-  gp.d = p->d;
-  gp.V = p->V;
-  gp.ldg = c.ldg;
-  gp.pl = reinterpret_cast<float*>(w + c.pl);
-  gp.pz = reinterpret_cast<float*>(w + c.pz);
-  gp.ps = reinterpret_cast<float*>(w + c.ps);
-  gp.tgt_c = tgt_c;
-  gp.zref = zref;
-  gp.live_rows = live_rows;
-  gp.dH = static_cast<__nv_bfloat16*>(dH);
-  gp.dW = dW;
-  gp.accumulate = 1;
-  gp.err = &state->status;
-  pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
-
-  // The ranges live on the device; the host enqueues the largest number of ranges the
-  // packing can produce and launches past the last range find no work.
-  for (int k = 0; k < c.max_ranges; ++k) {
-    const RangeRec* rg = ranges + k;
-    gp.range_ptr = &rg->row_begin;
-    gp.rowscale = nullptr;
-    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
-    if (rc != OAPL_OK) return rc;
-    merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
-                                         reinterpret_cast<float*>(w + c.ent_c), alpha, ztc, token_logp, state);
-    CKL();
-    seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp, seq_D, 1, &rg->seq_begin);
-    CKL();
-    coef_range_kernel<<<(p->S + 255) / 256, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, rg, p->P,
-                                                          p->beta_loss, p->loss_scale, coef);
-    CKL();
-    scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, alpha, lse, ztc, rg, p->d, p->V,
-                                                 c.ldg, Hs, rowscale, E);
-    CKL();
-    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
-    if (rc != OAPL_OK) return rc;
-    gp.rowscale = rowscale;
-    rc = launch_gemm<MODE_DH, 0, 1, 2>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
-    if (rc != OAPL_OK) return rc;
-  }
-  loss_kernel<<<1, 256, 0, st>>>(p->reward, p->group_id, vhat, seq_D, p->S, p->P, p->beta_loss,
-                                 p->loss_scale, coef, delta, loss, state);
+  group_advantage_kernel<<<(P + 7) / 8, 256, 0, st>>>(reward, group_id, S, P, eps, advantage);
   CKL();
   return OAPL_OK;
+}
+
+int oapl_grpo_loss_fwd_bwd(const oapl_problem* p, const float* logp_old, const float* advantage,
+                           float clip_eps, float* loss, float* seq_logp, float* token_logp, float* clip_frac,
+                           void* dH, float* dW, int accumulate_dW, void* ws, size_t ws_bytes, int flags,
+                           void* stream) {
+  int rc = check_problem(p, false);
+  if (rc != OAPL_OK) return rc;
+  if (!p->logp_inf || !logp_old || !advantage || !loss || !dH || !dW || !ws) return OAPL_ERR_INVALID_ARG;
+  if (!(clip_eps >= 0.f) || !std::isfinite(clip_eps) || !std::isfinite(p->loss_scale)) return OAPL_ERR_INVALID_ARG;
+  if (((uintptr_t)dH | (uintptr_t)dW) & 15) return OAPL_ERR_MISALIGNED;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, flags | OAPL_FLAG_FUSED, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  Objective ob;
+  memset(&ob, 0, sizeof(ob));
+  ob.grpo = true;
+  ob.logp_old = logp_old;
+  ob.adv = advantage;
+  ob.clip_eps = clip_eps;
+  ob.clip_frac = clip_frac;
+  return staged_fwd_bwd(p, ob, loss, seq_logp, token_logp, dH, dW, accumulate_dW, static_cast<uint8_t*>(ws), c,
+                        static_cast<cudaStream_t>(stream));
 }
 
 int oapl_entropy(const oapl_problem* p, float* token_entropy, float* seq_entropy, float* mean_entropy,

@@ -427,8 +427,10 @@ __global__ void coef_range_kernel(const float* __restrict__ reward, const int* _
 // this kernel writes Hs = bf16(s_n H_n), the row scales, and patches the target entries.
 // Rows between the range end and the next multiple of 256 get zero Hs rows (the dW
 // contraction reads whole 64-row slabs).  One warp per row.
+// The coefficient is the row's own (coef_row, token-level objectives) or its sequence's.
 __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const int* __restrict__ seq_c,
                                    const int* __restrict__ tgt_c, const float* __restrict__ coef,
+                                   const float* __restrict__ coef_row,
                                    const float* __restrict__ alpha, const float* __restrict__ lse,
                                    const float* __restrict__ ztc, const RangeRec* __restrict__ range,
                                    int d, int V, int ldg, __nv_bfloat16* __restrict__ Hs,
@@ -442,7 +444,7 @@ __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const i
     uint4* dst = reinterpret_cast<uint4*>(Hs + (size_t)i * d);
     if (i < re) {
       const float a = alpha[i];
-      const float s = -coef[seq_c[i]] * a;
+      const float s = -(coef_row ? coef_row[i] : coef[seq_c[i]]) * a;
       const uint4* src = reinterpret_cast<const uint4*>(Hc + (size_t)i * d);
       for (int k = lane; k < vec; k += 32) {
         uint4 x = src[k];
@@ -463,6 +465,120 @@ __global__ void scale_patch_kernel(const __nv_bfloat16* __restrict__ Hc, const i
     } else {
       for (int k = lane; k < vec; k += 32) dst[k] = make_uint4(0, 0, 0, 0);
     }
+  }
+}
+
+// =====================================================================================
+// GRPO with token-level importance weights (the paper's baseline objective, the display
+// in its Background section) on the same staged-exponential pipeline.
+// =====================================================================================
+// Group-normalised advantage: A_i = (r_i - mean_p) / (std_p + eps) over the members of the
+// sequence's group p (population standard deviation).  One warp per group, then the members
+// are written by the same warp.  A group without members writes nothing.
+__global__ void group_advantage_kernel(const float* __restrict__ reward, const int* __restrict__ group_id,
+                                       int S, int P, float eps, float* __restrict__ adv) {
+  const int p = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (p >= P) return;
+  double sum = 0.0;
+  int cnt = 0;
+  for (int i = lane; i < S; i += 32)
+    if (group_id[i] == p) { sum += (double)reward[i]; ++cnt; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  }
+  if (cnt == 0) return;
+  const double mean = sum / (double)cnt;
+  double ss = 0.0;
+  for (int i = lane; i < S; i += 32)
+    if (group_id[i] == p) { const double dlt = (double)reward[i] - mean; ss += dlt * dlt; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const double sd = sqrt(ss / (double)cnt);
+  for (int i = lane; i < S; i += 32)
+    if (group_id[i] == p) adv[i] = (float)(((double)reward[i] - mean) / (sd + (double)eps));
+}
+
+// Compaction of one more per-row float array (the previous policy's log-probs).
+__global__ void gather_f32_kernel(const float* __restrict__ src, const int* __restrict__ live_rows,
+                                  const DevState* st, float* __restrict__ dst) {
+  const int n_live = st->n_live;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_live; i += gridDim.x * blockDim.x)
+    dst[i] = src[live_rows[i]];
+}
+
+// One CTA per sequence of the range.  Per response token, with r = exp(lp - lp_old),
+// w = exp(lp_old - lp_inf) (data) and the sequence's advantage A:
+//     term  = w * min(r A, clip(r, 1-eps, 1+eps) A)
+//     coef  = dLoss/dlp = -lambda/|y| * w * A * r   where the unclipped branch is the minimum,
+//             0 where the clipped (constant) branch is.
+// Writes the per-row coefficients and, per sequence, (1/|y|) sum_t term and the number of
+// tokens on the clipped branch; fixed reduction order.
+__global__ void grpo_coef_kernel(const float* __restrict__ lp_c, const float* __restrict__ qold_c,
+                                 const float* __restrict__ qinf_c, const int* __restrict__ cstart,
+                                 const int* __restrict__ cend, const float* __restrict__ adv,
+                                 const int* __restrict__ seq_range, float clip_eps, float loss_scale,
+                                 float* __restrict__ coef_row, float* __restrict__ seq_obj,
+                                 int* __restrict__ seq_clipped) {
+  __shared__ double sh[8];
+  __shared__ int shc[8];
+  const int s = blockIdx.x;
+  if (s < seq_range[0] || s >= seq_range[1]) return;  // whole CTA
+  const int b = cstart[s], e = cend[s];
+  const double A = (double)adv[s];
+  const double inv_len = e > b ? 1.0 / (double)(e - b) : 0.0;
+  const double lo = 1.0 - (double)clip_eps, hi = 1.0 + (double)clip_eps;
+  double acc = 0.0;
+  int nclip = 0;
+  for (int i = b + threadIdx.x; i < e; i += blockDim.x) {
+    const double lp = (double)lp_c[i], lo_ = (double)qold_c[i];
+    const double r = exp(lp - lo_);
+    const double w = exp(lo_ - (double)qinf_c[i]);
+    const double rc = fmin(fmax(r, lo), hi);
+    const double t_un = r * A, t_cl = rc * A;
+    const bool unclipped = t_un <= t_cl;
+    acc += w * (unclipped ? t_un : t_cl);
+    nclip += unclipped ? 0 : 1;
+    coef_row[i] = unclipped ? (float)(-(double)loss_scale * inv_len * w * A * r) : 0.f;
+  }
+  acc = warp_sum_d(acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) nclip += __shfl_down_sync(0xffffffffu, nclip, o);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { sh[warp] = acc; shc[warp] = nclip; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    int n = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { t += sh[w]; n += shc[w]; }
+    seq_obj[s] = (float)(t * inv_len);
+    seq_clipped[s] = n;
+  }
+}
+
+// loss = -lambda * sum_i seq_obj[i];  clip_frac = clipped tokens / response tokens.
+__global__ void grpo_loss_kernel(const float* __restrict__ seq_obj, const int* __restrict__ seq_clipped,
+                                 int S, float loss_scale, float* __restrict__ loss,
+                                 float* __restrict__ clip_frac, DevState* st) {
+  __shared__ double sh[8];
+  __shared__ long long shc[8];
+  double acc = 0.0;
+  long long n = 0;
+  for (int i = threadIdx.x; i < S; i += blockDim.x) { acc += (double)seq_obj[i]; n += seq_clipped[i]; }
+  acc = warp_sum_d(acc);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) n += __shfl_down_sync(0xffffffffu, n, o);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) { sh[warp] = acc; shc[warp] = n; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    long long c = 0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) { t += sh[w]; c += shc[w]; }
+    *loss = (float)(-(double)loss_scale * t);
+    if (clip_frac) *clip_frac = st->n_live > 0 ? (float)((double)c / (double)st->n_live) : 0.f;
   }
 }
 

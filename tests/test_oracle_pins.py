@@ -341,3 +341,110 @@ def test_entropy_closed_forms_bounds_and_scipy():
         tot, cnt = tot + sum(vals), cnt + len(vals)
     assert mean == pytest.approx(tot / cnt, abs=1e-14)
     assert orc.sequence_entropy(ent, np.zeros(9, dtype=np.uint8), seq_id, 3)[1] == 0.0
+
+
+# ---------------------------------------------------------------- GRPO baseline
+def _grpo_problem(seed=0, noise=0.15):
+    r = np.random.default_rng(seed)
+    N, d, V, S, P = 14, 5, 9, 4, 2
+    H = r.normal(size=(N, d))
+    W = r.normal(size=(V, d)) * 0.6
+    targets = r.integers(0, V, size=N)
+    seq_id = np.sort(np.concatenate([np.arange(S), r.integers(0, S, size=N - S)]))
+    mask = np.ones(N, dtype=np.uint8)
+    for i in (0, 2):                       # a masked row in two sequences that keep other rows
+        rows = np.flatnonzero(seq_id == i)
+        if len(rows) > 1:
+            mask[rows[0]] = 0
+    mask[np.flatnonzero(seq_id == np.bincount(seq_id).argmax())[-1]] = 0
+    group_id = np.array([0, 0, 1, 1])
+    reward = np.array([1.0, 0.0, 0.5, 2.0])
+    lp, _ = orc.token_logprobs(H, W, targets, mask)
+    logp_old = lp + noise * r.normal(size=N)
+    logp_inf = logp_old + 0.1 * r.normal(size=N)
+    return dict(H=H, W=W, targets=targets, mask=mask, seq_id=seq_id, group_id=group_id, reward=reward,
+                logp_old=logp_old, logp_inf=logp_inf, S=S, P=P)
+
+
+def test_group_advantage_is_standardised_within_groups():
+    r = np.array([1.0, 0.0, 0.0, 1.0, 3.0, 3.0, 3.0, 7.0])
+    g = np.array([0, 0, 0, 0, 1, 1, 1, 2])
+    adv = orc.group_advantage(r, g, 4, 0.0 + 1e-12)
+    assert abs(adv[:4].mean()) < 1e-9 and adv[:4].std() == pytest.approx(1.0, abs=1e-9)
+    assert np.all(adv[4:7] == 0.0) and adv[7] == 0.0                  # equal rewards, singleton
+    # invariance to a positive affine map of the rewards (eps = 0 in the limit)
+    adv2 = orc.group_advantage(5.0 * r - 3.0, g, 4, 1e-12)
+    assert np.allclose(adv, adv2, atol=1e-9)
+    assert orc.group_advantage(r, g, 4, 1.0)[0] == pytest.approx(0.5 / (0.5 + 1.0))
+
+
+def test_grpo_loss_is_the_literal_display():
+    p = _grpo_problem(1, noise=0.3)
+    adv = orc.group_advantage(p["reward"], p["group_id"], p["P"], 1e-6)
+    out = orc.grpo_fwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], p["logp_old"], p["logp_inf"],
+                       adv, p["S"], 0.2, 0.25)
+    # the display, typed out: 1/|y| sum_t  IS ratio * min(r A, clip(r) A), summed over rollouts
+    z = p["H"] @ p["W"].T
+    lsm = z - scipy.special.logsumexp(z, axis=1, keepdims=True)
+    J = 0.0
+    for i in range(p["S"]):
+        rows = [n for n in range(len(p["mask"])) if p["mask"][n] and p["seq_id"][n] == i]
+        acc = 0.0
+        for n in rows:
+            pi, pi_old, pi_vllm = (math.exp(lsm[n, p["targets"][n]]), math.exp(p["logp_old"][n]),
+                                   math.exp(p["logp_inf"][n]))
+            r_t = pi / pi_old
+            acc += (pi_old / pi_vllm) * min(r_t * adv[i], float(np.clip(r_t, 0.8, 1.2)) * adv[i])
+        J += acc / len(rows)
+    assert out["loss"] == pytest.approx(-0.25 * J, rel=1e-12)
+    assert 0 < out["clipped"].sum() < p["mask"].sum()                 # both branches are exercised
+
+
+def test_grpo_on_policy_reduces_to_the_policy_gradient():
+    # pi_old = pi and pi_vllm = pi_old: every ratio is 1, nothing is clipped, the loss is
+    # -lambda sum_i A_i (zero for standardised advantages) and dloss/dlp_t = -lambda A_i / |y_i|
+    p = _grpo_problem(2)
+    lp, _ = orc.token_logprobs(p["H"], p["W"], p["targets"], p["mask"])
+    adv = orc.group_advantage(p["reward"], p["group_id"], p["P"], 1e-9)
+    out = orc.grpo_from_logprobs(lp, lp, lp, p["mask"], p["seq_id"], adv, p["S"], 0.2, 1.0)
+    assert abs(out["loss"]) < 1e-9 and not out["clipped"].any()
+    for n in np.flatnonzero(p["mask"]):
+        i = p["seq_id"][n]
+        assert out["coef"][n] == pytest.approx(-adv[i] / out["T"][i], rel=1e-12)
+
+
+def test_grpo_clipped_tokens_are_constant():
+    p = _grpo_problem(3, noise=0.0)
+    lp, _ = orc.token_logprobs(p["H"], p["W"], p["targets"], p["mask"])
+    adv = np.array([1.0, -1.0, 1.0, -1.0])
+    old = lp.copy()
+    old[p["seq_id"] == 0] -= 0.5       # r = e^0.5 > 1.2 with A > 0: clipped at (1+eps) A
+    old[p["seq_id"] == 1] += 0.5       # r = e^-0.5 < 0.8 with A < 0: clipped at (1-eps) A
+    old[p["seq_id"] == 2] += 0.5       # r < 0.8 with A > 0: unclipped
+    old[p["seq_id"] == 3] -= 0.5       # r > 1.2 with A < 0: unclipped
+    out = orc.grpo_from_logprobs(lp, old, old, p["mask"], p["seq_id"], adv, p["S"], 0.2, 1.0)
+    live = p["mask"].astype(bool)
+    assert out["clipped"][live & (p["seq_id"] <= 1)].all() and not out["clipped"][live & (p["seq_id"] >= 2)].any()
+    assert np.all(out["coef"][p["seq_id"] <= 1] == 0.0)
+    want = -(1.2 * 1.0 + 0.8 * -1.0 + math.exp(-0.5) * 1.0 + math.exp(0.5) * -1.0)
+    assert out["loss"] == pytest.approx(want, rel=1e-12)
+
+
+def test_grpo_gradient_matches_central_differences():
+    p = _grpo_problem(4)
+    adv = orc.group_advantage(p["reward"], p["group_id"], p["P"], 1e-6)
+    f = lambda H, W: orc.grpo_fwd(H, W, p["targets"], p["mask"], p["seq_id"], p["logp_old"], p["logp_inf"],
+                                  adv, p["S"], 0.2, 0.5)
+    out = f(p["H"], p["W"])
+    assert np.abs(np.abs(out["ratio"][p["mask"] == 1] - 1.0) - 0.2).min() > 1e-3   # away from the kinks
+    dH, dW = orc.token_coef_bwd(p["H"], p["W"], p["targets"], p["mask"], out["coef"])
+    h = 1e-6
+    for X, dX, name in ((p["H"], dH, "H"), (p["W"], dW, "W")):
+        for idx in np.ndindex(X.shape):
+            Xp, Xm = X.copy(), X.copy()
+            Xp[idx] += h
+            Xm[idx] -= h
+            num = ((f(Xp, p["W"]) if name == "H" else f(p["H"], Xp))["loss"] -
+                   (f(Xm, p["W"]) if name == "H" else f(p["H"], Xm))["loss"]) / (2 * h)
+            assert num == pytest.approx(dX[idx], rel=2e-5, abs=2e-8), (name, idx)
+    assert np.all(dH[p["mask"] == 0] == 0.0)
