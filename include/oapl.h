@@ -176,6 +176,27 @@ int oapl_grpo_loss_fwd_bwd(const oapl_problem* problem /*host*/, const float* lo
                            void* ws, size_t ws_bytes, int flags, void* stream);
 
 /*
+ * The optimizer step that follows the gradient in a trainer step, for the LM-head weight:
+ * AdamW with gradient clipping by norm, the optimizer of the paper's "Experimental Details"
+ * tables (math: lr 1e-6, betas 0.9/0.95, weight decay 1e-2, clip threshold 1e-3; code
+ * generation: betas 0.9/0.999, threshold 1.0).  With g = dW * min(1, clip_norm / (||grad|| + 1e-6)),
+ * where ||grad||^2 = sum(dW^2) + *other_sq_norm (the squared gradient norm of the model's other
+ * parameters, device scalar or NULL), step t >= 1:
+ *     m = beta1 m + (1-beta1) g;   v = beta2 v + (1-beta2) g^2;
+ *     theta = theta (1 - lr weight_decay) - lr (m / (1-beta1^t)) / (sqrt(v / (1-beta2^t)) + eps).
+ * theta is the fp32 `master` copy [n] when given (W then receives its bf16 rounding), else the
+ * bf16 W itself.  W [n] bf16 (8-byte aligned), dW / m / v / master [n] f32 (16-byte aligned),
+ * all updated in place; n = V*d.  clip_norm <= 0 disables clipping.  grad_norm [1] or NULL
+ * receives ||grad||.  ws: oapl_adamw_workspace_bytes() bytes of device scratch (partial sums).
+ * Two HBM-bound passes: dW is read twice, every other array once (34 bytes per element with a
+ * master copy).
+ */
+size_t oapl_adamw_workspace_bytes(void);
+int oapl_adamw_step(void* W, float* master, const float* dW, float* m, float* v, int64_t n, int64_t step,
+                    float lr, float beta1, float beta2, float eps, float weight_decay, float clip_norm,
+                    const float* other_sq_norm, float* grad_norm, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Policy entropy of the trainer policy on the response tokens, the training-dynamics
  * diagnostic of the paper's experiments (the entropy curves of OAPL against GRPO in the
  * "Training dynamics" figure and the "sequence entropy" discussed beside it):

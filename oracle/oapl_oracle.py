@@ -268,6 +268,28 @@ def token_coef_bwd(H, W, targets, mask, coef_tok):
     return loss_bwd(H, W, targets, mask, np.arange(n), coef_tok)
 
 
+# --------------------------------------------------------------------------
+# the optimizer step of the paper's hyper-parameter tables: AdamW with
+# gradient clipping by norm (decoupled weight decay, Loshchilov & Hutter)
+# --------------------------------------------------------------------------
+def adamw_step(theta, grad, m, v, step, lr, beta1, beta2, eps, weight_decay, clip_norm, other_sq_norm=0.0):
+    """One AdamW step on float64 arrays; returns (theta, m, v, grad_norm).
+
+    The gradient is first scaled by min(1, clip_norm / (||grad|| + 1e-6)) with
+    ||grad||^2 = sum(grad^2) + other_sq_norm (clip_norm <= 0: no clipping)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    g = np.asarray(grad, dtype=np.float64)
+    norm = float(np.sqrt((g * g).sum() + other_sq_norm))
+    if clip_norm > 0:
+        g = g * min(1.0, clip_norm / (norm + 1e-6))
+    m = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    mhat = m / (1.0 - beta1 ** step)
+    vhat = v / (1.0 - beta2 ** step)
+    theta = theta * (1.0 - lr * weight_decay) - lr * mhat / (np.sqrt(vhat) + eps)
+    return theta, m, v, norm
+
+
 def token_entropy(H, W, mask):
     """Per-row policy entropy -sum_v p ln p (the diagnostic tracked in the
     paper's entropy figure); 0 on masked rows."""

@@ -23,7 +23,7 @@ EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
            "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy", "oapl_group_advantage",
-           "oapl_grpo_loss_fwd_bwd"]
+           "oapl_grpo_loss_fwd_bwd", "oapl_adamw_workspace_bytes", "oapl_adamw_step"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.oapl_group_advantage.argtypes = [vp, vp, ctypes.c_int32, ctypes.c_int32, f32, vp, vp]
         L.oapl_grpo_loss_fwd_bwd.restype = i32
         L.oapl_grpo_loss_fwd_bwd.argtypes = [pp, vp, vp, f32, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
+        L.oapl_adamw_workspace_bytes.restype = sz
+        L.oapl_adamw_workspace_bytes.argtypes = []
+        L.oapl_adamw_step.restype = i32
+        L.oapl_adamw_step.argtypes = [vp, vp, vp, vp, vp, i64, i64, f32, f32, f32, f32, f32, f32, vp, vp, vp, sz, vp]
         L.oapl_entropy.restype = i32
         L.oapl_entropy.argtypes = [pp, vp, vp, vp, vp, sz, i32, vp]
         L.oapl_profile_enable.restype = i32
@@ -187,6 +191,18 @@ def oapl_grpo_loss_fwd_bwd(problem, logp_old, advantage, clip_eps, loss, seq_log
                                       _ptr(dW), int(accumulate_dW), _ptr(ws), ws.numel(), flags, _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_grpo_loss_fwd_bwd")
+
+
+def oapl_adamw_step(W, master, dW, m, v, step, lr, beta1, beta2, eps, weight_decay, clip_norm,
+                    other_sq_norm=None, grad_norm=None, ws=None):
+    if ws is None:
+        ws = torch.empty(int(lib().oapl_adamw_workspace_bytes()), dtype=torch.uint8, device=W.device)
+    rc = lib().oapl_adamw_step(_ptr(W), _ptr(master), _ptr(dW), _ptr(m), _ptr(v), W.numel(), int(step), lr, beta1,
+                               beta2, eps, weight_decay, clip_norm, _ptr(other_sq_norm), _ptr(grad_norm), _ptr(ws),
+                               ws.numel(), _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_adamw_step")
+    return ws
 
 
 def oapl_entropy(problem, token_entropy, seq_entropy, mean_entropy, ws, flags=0):

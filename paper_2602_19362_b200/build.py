@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liboapl.so")
 SOURCES = ["oapl_api.cu"]
-DEPS = ["oapl_api.cu", "gemm_sm100.cuh", "small_kernels.cuh", "sm100_ptx.cuh",
+DEPS = ["oapl_api.cu", "gemm_sm100.cuh", "small_kernels.cuh", "sm100_ptx.cuh", "sweep_schedule.cuh", "adamw.cuh",
         os.path.join("..", "..", "include", "oapl.h")]
 
 

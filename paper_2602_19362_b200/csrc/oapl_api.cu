@@ -10,6 +10,7 @@
 #include <cstring>
 
 #include "../../include/oapl.h"
+#include "adamw.cuh"
 #include "gemm_sm100.cuh"
 #include "small_kernels.cuh"
 
@@ -682,6 +683,45 @@ int oapl_grpo_loss_fwd_bwd(const oapl_problem* p, const float* logp_old, const f
   ob.clip_frac = clip_frac;
   return staged_fwd_bwd(p, ob, loss, seq_logp, token_logp, dH, dW, accumulate_dW, static_cast<uint8_t*>(ws), c,
                         static_cast<cudaStream_t>(stream));
+}
+
+size_t oapl_adamw_workspace_bytes(void) { return sizeof(double) * kAdamMaxPartials; }
+
+int oapl_adamw_step(void* W, float* master, const float* dW, float* m, float* v, int64_t n, int64_t step,
+                    float lr, float beta1, float beta2, float eps, float weight_decay, float clip_norm,
+                    const float* other_sq_norm, float* grad_norm, void* ws, size_t ws_bytes, void* stream) {
+  if (!W || !dW || !m || !v || !ws || n <= 0 || step < 1) return OAPL_ERR_INVALID_ARG;
+  if (!(lr >= 0.f) || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps >= 0.f) ||
+      !(weight_decay >= 0.f) || !std::isfinite(lr) || !std::isfinite(eps) || !std::isfinite(weight_decay) ||
+      !std::isfinite(clip_norm))
+    return OAPL_ERR_INVALID_ARG;
+  if (((uintptr_t)W & 7) || (((uintptr_t)dW | (uintptr_t)m | (uintptr_t)v | (uintptr_t)master) & 15) ||
+      ((uintptr_t)ws & 7))
+    return OAPL_ERR_MISALIGNED;
+  if (ws_bytes < sizeof(double) * kAdamMaxPartials) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  const int n_sm = sm_count();
+  if (n_sm <= 0) return OAPL_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  double* partial = static_cast<double*>(ws);
+  const size_t work = ((size_t)n / 4 + kAdamThreads - 1) / kAdamThreads;
+  int grid = n_sm * 8;
+  if ((size_t)grid > work) grid = work ? (int)work : 1;
+  if (grid > kAdamMaxPartials) grid = kAdamMaxPartials;
+  sqnorm_partial_kernel<<<grid, kAdamThreads, 0, st>>>(dW, (size_t)n, partial);
+  CKL();
+  AdamParams a;
+  a.lr = lr;
+  a.beta1 = beta1;
+  a.beta2 = beta2;
+  a.eps = eps;
+  a.weight_decay = weight_decay;
+  a.clip_norm = clip_norm;
+  a.bias1 = (float)(1.0 - std::pow((double)beta1, (double)step));
+  a.bias2 = (float)(1.0 - std::pow((double)beta2, (double)step));
+  adamw_kernel<<<grid, kAdamThreads, 0, st>>>(dW, m, v, master, static_cast<__nv_bfloat16*>(W), (size_t)n, partial,
+                                              grid, other_sq_norm, a, grad_norm);
+  CKL();
+  return OAPL_OK;
 }
 
 int oapl_entropy(const oapl_problem* p, float* token_entropy, float* seq_entropy, float* mean_entropy,

@@ -448,3 +448,45 @@ def test_grpo_gradient_matches_central_differences():
                    (f(Xm, p["W"]) if name == "H" else f(p["H"], Xm))["loss"]) / (2 * h)
             assert num == pytest.approx(dX[idx], rel=2e-5, abs=2e-8), (name, idx)
     assert np.all(dH[p["mask"] == 0] == 0.0)
+
+
+# ---------------------------------------------------------------- AdamW + clipping by norm
+def test_adamw_matches_torch_optimizer_and_clip_grad_norm():
+    import torch
+    r = np.random.default_rng(11)
+    theta0 = r.normal(size=(37,)) * 0.02
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=1e-2)
+    p = torch.nn.Parameter(torch.tensor(theta0, dtype=torch.float64))
+    opt = torch.optim.AdamW([p], lr=hp["lr"], betas=(hp["beta1"], hp["beta2"]), eps=hp["eps"],
+                            weight_decay=hp["weight_decay"])
+    theta, m, v = theta0.copy(), np.zeros(37), np.zeros(37)
+    for step in range(1, 6):
+        g = r.normal(size=37) * (10.0 if step % 2 else 1e-3)       # clipped and unclipped steps
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        torch.nn.utils.clip_grad_norm_([p], max_norm=1.0)
+        opt.step()
+        theta, m, v, norm = orc.adamw_step(theta, g, m, v, step, clip_norm=1.0, **hp)
+        assert norm == pytest.approx(np.linalg.norm(g), rel=1e-14)
+        assert np.allclose(theta, p.detach().numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_adamw_closed_forms():
+    g = np.array([3.0, -0.5, 2.0, -4.0])
+    th = np.array([1.0, -2.0, 0.5, 0.25])
+    z = np.zeros(4)
+    # first step, no decay, eps = 0: the bias-corrected ratio is sign(g), whatever the gradient's scale,
+    # so clipping cannot change it
+    a, _, _, _ = orc.adamw_step(th, g, z, z, 1, 1e-2, 0.9, 0.95, 0.0, 0.0, 0.0)
+    assert np.allclose(a, th - 1e-2 * np.sign(g), atol=1e-15)
+    b, _, _, _ = orc.adamw_step(th, g, z, z, 1, 1e-2, 0.9, 0.95, 0.0, 0.0, 1e-3)
+    assert np.allclose(a, b, atol=1e-12)
+    # zero gradient: decoupled weight decay only
+    c, m, v, norm = orc.adamw_step(th, z, z, z, 1, 1e-2, 0.9, 0.95, 1e-8, 0.1, 1.0)
+    assert np.allclose(c, th * (1 - 1e-3), atol=1e-15) and norm == 0.0 and not m.any() and not v.any()
+    # the clipped gradient has norm clip_norm (up to the 1e-6 guard): read it off m after one step
+    _, m, _, norm = orc.adamw_step(th, g, z, z, 1, 1e-2, 0.9, 0.95, 1e-8, 0.0, 0.5)
+    assert np.linalg.norm(m / 0.1) == pytest.approx(0.5, rel=1e-5) and norm == pytest.approx(np.linalg.norm(g))
+    # other parameters' gradient norm enters the clip factor
+    _, m2, _, norm2 = orc.adamw_step(th, g, z, z, 1, 1e-2, 0.9, 0.95, 1e-8, 0.0, 0.5, other_sq_norm=100.0)
+    assert norm2 == pytest.approx(math.sqrt((g * g).sum() + 100.0))
+    assert np.allclose(m2, 0.1 * g * 0.5 / (norm2 + 1e-6), rtol=1e-12)
