@@ -176,7 +176,7 @@ def run_reference(args) -> None:
 def run_cuda(args) -> None:
     import torch
     import torch.distributed as dist
-    from paper_2602_19362_b200 import binding as B, synth
+    from paper_2602_19362_b200 import binding as B, dp, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -205,7 +205,8 @@ def run_cuda(args) -> None:
     batch = synth.make_batch(wl, seed=args.seed + rank, device=str(dev), beta=args.beta)
     N, S, P, d, V = (batch[k] for k in ("N", "S", "P", "d", "V"))
     n_live = batch["live_tokens"]
-    prob = B.make_problem(batch)
+    # the loss normalises over the rollouts of all ranks
+    prob = B.make_problem(batch, loss_scale=1.0 / (S * world))
     fused = args.path == "single-call"
     ws = B.alloc_workspace(prob, B.OAPL_FLAG_FUSED if fused else 0, device=dev)
     loss = torch.zeros(1, device=dev)
@@ -228,6 +229,12 @@ def run_cuda(args) -> None:
         clip_frac = torch.zeros(1, device=dev)
 
     def step():
+        local_step()
+        if world > 1:
+            # the one exchange of the data-parallel step: sum of dW (and of the loss) over the ranks
+            dp.allreduce_outputs(loss, dW)
+
+    def local_step():
         if grpo:
             B.oapl_grpo_loss_fwd_bwd(prob, logp_old, adv, 0.2, loss, seq_logp, None, clip_frac, dH, dW, False, ws)
         elif fused:
@@ -370,7 +377,7 @@ def run_cuda(args) -> None:
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{wl.name}-scale: d={d}, V={V}, {P} prompts x {wl.samples} rollouts, "
                                    f"lengths {wl.length}, padded_to={wl.padded_to}, beta={batch['beta_v']}",
-                       "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts",
+                       "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts" + (", NCCL all-reduce of dW and loss in the step" if world > 1 else ""),
                        "l2": "inputs larger than L2 (H, W, g chunk each > 126 MB); no flush needed",
                        "api": ("oapl_grpo_loss_fwd_bwd" if grpo else "oapl_loss_fwd_bwd") if fused
                               else "oapl_loss_fwd + oapl_loss_bwd",

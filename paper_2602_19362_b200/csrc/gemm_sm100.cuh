@@ -94,7 +94,59 @@ struct GemmParams {
   int* err;  // device status word
   // optional timing: {SM cycles, nanoseconds} of CTA 0, added up per launch (null = off)
   unsigned long long* clk;
+  // Lock-step of the CTA pairs (null / 0 = off): every sync_every K-steps the pairs meet at a
+  // counter in global memory, so that pairs reading the same operand slabs stay within the
+  // time those slabs live in L2.  The counter must be zero at launch.
+  unsigned int* sync_ctr;
+  int sync_every;
 };
+
+// Largest number of K-steps any CTA pair of this launch executes (all pairs compute the same
+// value): it fixes how many lock-step meetings a pair that runs out of tiles early must still
+// be counted for.
+template <int MODE, int NACC>
+__device__ __forceinline__ long long max_ksteps_per_pair(const GemmParams& p, int row_begin, int row_end) {
+  constexpr int kTN = NACC * kBN;
+  const int rows = row_end - row_begin;
+  const int npairs = gridDim.x >> 1;
+  if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
+    if (rows <= 0) return 0;
+    const int VT = (p.V + kBN - 1) / kBN;
+    const int nrb = (rows + kTileM - 1) / kTileM;
+    const SweepShape sh = sweep_shape(nrb, p.R, p.C, VT);
+    long long tiles = (long long)sh.nfull * ((VT + p.C - 1) / p.C);
+    if (sh.rem) tiles += (VT + sh.Ct - 1) / sh.Ct;
+    return tiles * (p.d / kBK);
+  }
+  long long tiles, nk;
+  if (MODE == MODE_DH) {
+    if (rows <= 0) return 0;
+    tiles = (long long)((rows + kTileM - 1) / kTileM) * ((p.d + kTN - 1) / kTN);
+    nk = (p.V + kBK - 1) / kBK;
+  } else if (MODE == MODE_DW) {
+    if (rows <= 0) return 0;
+    tiles = (long long)((p.V + kTileM - 1) / kTileM) * ((p.d + kTN - 1) / kTN);
+    nk = (rows + kBK - 1) / kBK;
+  } else {
+    tiles = (long long)((p.M + kTileM - 1) / kTileM) * ((p.N + kTN - 1) / kTN);
+    nk = p.K / kBK;
+  }
+  return ((tiles + npairs - 1) / npairs) * nk;
+}
+
+// One meeting of the lock-step: count this pair in and wait (bounded) until all pairs of the
+// launch have been counted `epoch` times.  Returns false when the wait gave up: the caller then
+// stops meeting (the others give up once as well); results do not depend on the meetings.
+__device__ __forceinline__ bool lockstep_meet(unsigned int* ctr, unsigned int target) {
+  atomicAdd(ctr, 1u);
+  volatile unsigned int* v = ctr;
+  if (*v >= target) return true;
+  const unsigned long long t0 = global_timer_ns();
+  while (*v < target) {
+    if (global_timer_ns() - t0 > 200000ull) return false;  // 200 us
+  }
+  return true;
+}
 
 struct Tile {
   int m0, n0;    // tile origin (A's M coordinate, B's N coordinate)
@@ -286,8 +338,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       Tile t;
       bool ok = true;
+      // the leader CTA's producer keeps the pair in step with the other pairs (its partner
+      // follows through the shared pipeline barriers)
+      bool meet = p.sync_ctr != nullptr && p.sync_every > 0 && rank == 0;
+      const unsigned int npairs = gridDim.x >> 1;
+      unsigned int epochs = 0;
       for (int j = 0; ok && get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
         for (int kb = 0; kb < t.nk; ++kb, ++it) {
+          if (meet && it % (uint32_t)p.sync_every == 0) {
+            ++epochs;
+            meet = lockstep_meet(p.sync_ctr, epochs * npairs);
+          }
           const int s = it % kStages;
           if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag)) {
             ok = false;
@@ -321,6 +382,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           }
         }
+      }
+      if (meet) {
+        // out of tiles: be counted for the meetings the longest-running pair still holds
+        const long long mx = max_ksteps_per_pair<MODE, NACC>(p, row_begin, row_end);
+        const long long total = (mx + p.sync_every - 1) / p.sync_every;
+        if (total > (long long)epochs) atomicAdd(p.sync_ctr, (unsigned int)(total - epochs));
       }
     }
   } else if (warp == 1) {

@@ -21,11 +21,12 @@ static std::atomic<uint64_t> g_launches{0};
 
 constexpr int kChunkRowsDefault = 74 * 128;  // half of a 148-SM wave of row blocks
 constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref) in the single-call path
+constexpr int kSyncSlots = 4096;             // lock-step counters in the workspace, one per contraction launch
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Carve {
-  size_t state, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, ent_c, pm, pl, pz, ps, cstart,
+  size_t state, sync, block_cnt, block_off, live_rows, tgt_c, seq_c, q_c, lp_c, lse, ent_c, pm, pl, pz, ps, cstart,
       cend, seq_D, coef, vhat, seq_logp, Hc, G, zref, alpha, ztc, rowscale, Hs, ranges, coef_row, qo_c,
       seq_obj, seq_clip, total;
   int n_pad, nblk, chunk_rows, ldg;
@@ -56,6 +57,7 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
     return o;
   };
   c->state = take(sizeof(DevState));
+  c->sync = take(4 * (size_t)kSyncSlots);
   c->block_cnt = take(4 * (size_t)c->nblk);
   c->block_off = take(4 * (size_t)c->nblk);
   c->live_rows = take(4 * n_pad);
@@ -168,6 +170,20 @@ static void pick_sweep(int n_sm, int d, int vtiles, int* R, int* C) {
   *C = c;
 }
 
+// Lock-step meetings of the CTA pairs of one contraction launch (see GemmParams::sync_ctr):
+// counter number `slot` of the workspace, which the caller has zeroed; every `nk_tile`-aligned
+// 32 K-steps or so.  OAPL_SYNC_EVERY overrides the interval (0 switches the meetings off).
+static void set_lockstep(GemmParams* gp, uint8_t* ws, const Carve& c, int slot, int nk_tile) {
+  static const int forced = env_int("OAPL_SYNC_EVERY", -1);
+  gp->sync_ctr = nullptr;
+  gp->sync_every = 0;
+  if (forced == 0 || slot < 0 || slot >= kSyncSlots) return;
+  int every = forced > 0 ? forced : 32;
+  if (nk_tile > 0) every = ((every + nk_tile - 1) / nk_tile) * nk_tile;  // whole tiles of a sweep
+  gp->sync_ctr = reinterpret_cast<unsigned int*>(ws + c.sync) + slot;
+  gp->sync_every = every;
+}
+
 // Optional per-contraction timing (off by default): an event pair around every
 // contraction launch, summed per kind by oapl_profile_read.
 constexpr int kProfSlots = 2048;
@@ -263,6 +279,7 @@ static int prologue(const oapl_problem* p, const Carve& c, uint8_t* ws, float* t
   __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + c.Hc);
 
   CK(cudaMemsetAsync(state, 0, sizeof(DevState), st));
+  CK(cudaMemsetAsync(ws + c.sync, 0, 4 * (size_t)kSyncSlots, st));
   CK(cudaMemsetAsync(cstart, 0, 4 * (size_t)p->S, st));
   CK(cudaMemsetAsync(cend, 0, 4 * (size_t)p->S, st));
   if (token_logp) CK(cudaMemsetAsync(token_logp, 0, 4 * (size_t)p->N, st));
@@ -318,6 +335,7 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.ps = reinterpret_cast<float*>(ws + c.ps);
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
+  set_lockstep(&gp, ws, c, 0, p->d / kBK);
   int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
@@ -431,6 +449,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
     const RangeRec* rg = ranges + k;
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
+    set_lockstep(&gp, w, c, 3 * k, p->d / kBK);
     rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
     merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
@@ -450,9 +469,11 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
     scale_patch_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, seq_c, tgt_c, coef, ob.grpo ? coef_row : nullptr, alpha,
                                                  lse, ztc, rg, p->d, p->V, c.ldg, Hs, rowscale, E);
     CKL();
+    set_lockstep(&gp, w, c, 3 * k + 1, 0);
     rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
     gp.rowscale = rowscale;
+    set_lockstep(&gp, w, c, 3 * k + 2, 0);
     rc = launch_gemm<MODE_DH, 0, 1, 2>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
@@ -619,12 +640,17 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   // Row chunks of the compacted rows.  The live-row count lives on the device, so the
   // host enqueues every chunk the row count N could need; chunks past the live rows
   // find no tile and return at once.
+  CK(cudaMemsetAsync(w + c.sync, 0, 4 * (size_t)kSyncSlots, st));
+  int slot = 0;
   for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
     gp.row_begin = r0;
+    set_lockstep(&gp, w, c, slot++, p->d / kBK);
     rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
+    set_lockstep(&gp, w, c, slot++, 0);
     rc = launch_gemm<MODE_DH, 0, 1, 2>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
+    set_lockstep(&gp, w, c, slot++, 0);
     rc = launch_gemm<MODE_DW, 1, 1, 2>(tmGmn, tmHmn, tmGmn, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
@@ -842,7 +868,7 @@ constexpr int kStaticMaxRows = 2048;
 constexpr int kStaticMaxD = 1024;
 constexpr int kStaticMaxSeq = 2048;
 constexpr size_t kStaticScratchBytes =
-    1024 /*state*/ + 2 * 1024 /*block counts, offsets*/ + 7 * 4 * (size_t)kStaticMaxRows /*per-row arrays*/ +
+    1024 /*state*/ + 4 * kSyncSlots /*lock-step counters*/ + 2 * 1024 /*block counts, offsets*/ + 7 * 4 * (size_t)kStaticMaxRows /*per-row arrays*/ +
     4 * 4 * (size_t)kStaticMaxRows * kMaxSplits /*log-sum-exp partials*/ +
     3 * 4 * (size_t)kStaticMaxSeq /*per-sequence arrays*/ +
     2 * (size_t)kStaticMaxRows * kStaticMaxD /*compacted H*/ + 16 * 1024 /*alignment slack*/;
@@ -896,6 +922,7 @@ int oapl_token_logprobs_static(const oapl_problem* p, float* token_logp, float* 
     return o;
   };
   c.state = take(sizeof(DevState));
+  c.sync = take(4 * (size_t)kSyncSlots);
   c.block_cnt = take(4 * (size_t)c.nblk);
   c.block_off = take(4 * (size_t)c.nblk);
   c.live_rows = take(4 * n_pad);

@@ -3,6 +3,7 @@ per-rank times, sum of the per-rank token counts)."""
 import os
 import sys
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -40,3 +41,56 @@ def test_identity_without_process_group():
     import bench
     assert bench.reduce_max(3.5, None, "cpu") == 3.5
     assert bench.reduce_sum(7.0, None, "cpu") == 7.0
+
+
+def _dp_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import oapl_oracle as orc
+    from paper_2602_19362_b200 import dp, synth
+    from tests import helpers_cpu as hc
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    full = synth.make_batch(hc.DP_WORKLOAD, seed=3)
+    shard = dp.shard_by_prompt(full, rank, world)
+    ref = hc.oracle_step(shard)
+    loss = torch.tensor([ref["loss"]], dtype=torch.float64)
+    dW = torch.from_numpy(ref["dW"])
+    dp.allreduce_outputs(loss, dW)
+    q.put((rank, float(loss), dW.numpy(), shard["N"], shard["S"], shard["P"], ref["dH"], np.asarray(ref["vhat"])))
+    dist.destroy_process_group()
+
+
+def test_sharding_by_prompt_plus_allreduce_reproduces_the_single_rank_step():
+    # Eq. 2 / Eq. 3 couple only rollouts of one prompt: two ranks holding whole groups, with the
+    # global loss_scale, must sum to the one-rank loss and dW; dH rows stay with their rank
+    import numpy as np
+    from paper_2602_19362_b200 import dp, synth
+    from tests import helpers_cpu as hc
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_dp_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted((q.get(timeout=300) for _ in procs), key=lambda t: t[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    full = synth.make_batch(hc.DP_WORKLOAD, seed=3)
+    ref = hc.oracle_step(full)
+    for rank, loss, dW, N, S, P, dH, vhat in got:
+        assert loss == pytest.approx(ref["loss"], rel=1e-12)
+        assert np.allclose(dW, ref["dW"], rtol=1e-10, atol=1e-14)
+    assert sum(g[3] for g in got) == full["N"] and sum(g[4] for g in got) == full["S"]
+    assert sum(g[5] for g in got) == full["P"]
+    assert np.allclose(np.concatenate([g[6] for g in got]), ref["dH"], rtol=1e-10, atol=1e-14)
+    assert np.allclose(np.concatenate([g[7] for g in got]), ref["vhat"], rtol=1e-12)
+
+
+def test_prompt_blocks_cover_every_prompt_once():
+    from paper_2602_19362_b200 import dp
+    for P, world in ((16, 8), (7, 3), (4, 4), (3, 5)):
+        owned = [list(dp.prompts_of_rank(P, r, world)) for r in range(world)]
+        assert sorted(sum(owned, [])) == list(range(P))
+        assert max(map(len, owned)) - min(map(len, owned)) <= 1
