@@ -26,6 +26,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "response tokens/sec for OAPL loss fwd+bwd"
+MEASURED_DRAM_BYTES_PER_STEP = 794.4e9
 UNIT = "tokens/s"
 
 
@@ -363,7 +364,12 @@ def run_cuda(args) -> None:
     roofline = {"bound": "tensor", "kernel": "gemm_kernel (tcgen05, one template: " + ("lse_e|dW|dH)" if fused else "lse|grad|dH|dW)"),
                 "executed_flops_per_step": exec_factor * n_live * d * V,
                 "achieved": exec_tflops, "peak": peak, "unit": "TFLOP/s",
-                "frac": exec_tflops / peak if exec_tflops else None, "traffic": None,
+                "frac": exec_tflops / peak if exec_tflops else None,
+                # DRAM bytes of the contraction launches of one step of this workload
+                # (dram__bytes_read.sum + dram__bytes_write.sum, one ncu pass over the 102 launches of a
+                # step; profiles/gemm_kernel_7b.md); only valid for the default workload and path
+                "traffic": MEASURED_DRAM_BYTES_PER_STEP if (fused and not grpo and args.workload == "7b"
+                                                            and not (args.prompts or args.samples)) else None,
                 "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
                 "credited_tflops": flops_step / (ms_step * 1e-3) / 1e12,
                 "credited_frac_of_sustained": flops_step / (ms_step * 1e-3) / 1e12 / peaks["sustained"],
@@ -399,7 +405,7 @@ def main() -> None:
     ap.add_argument("--workload", default="7b")
     ap.add_argument("--beta", type=float, default=1.0)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--ref-rows", type=int, default=256, help="response tokens in the CPU oracle sample")
+    ap.add_argument("--ref-rows", type=int, default=2048, help="response tokens in the CPU oracle sample")
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (profiling)")
     ap.add_argument("--samples", type=int, default=0, help="override rollouts per prompt (profiling)")
     ap.add_argument("--path", default="single-call", choices=["single-call", "two-calls"],
