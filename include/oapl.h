@@ -131,7 +131,7 @@ int oapl_loss_bwd(const oapl_problem* problem /*host*/, void* dH, float* dW, int
  * dH = rowscale(e'.W), dW += e'^T.(scaled H).  Executed work is 6*N*d*V flops instead of 8.
  *
  * Workspace: oapl_workspace_bytes(problem, OAPL_FLAG_FUSED).  It holds e for 32768 rows
- * (2 bytes * round_up(V,256) each; OAPL_STAGE_ROWS in the environment changes the count), so
+ * (2 bytes * round_up(V,512) each; OAPL_STAGE_ROWS in the environment changes the count), so
  * it does not grow with N*V; a sequence with more live rows than that cannot be staged and
  * raises OAPL_ERR_SEQUENCE_TOO_LONG in the status word (outputs are then not meaningful;
  * use the two separate calls).  A target whose probability under the policy is below

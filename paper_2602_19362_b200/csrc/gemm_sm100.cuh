@@ -24,8 +24,14 @@
 //   NACC = 2  256 x 512 pair tile: both accumulators belong to one tile and every A slab
 //             feeds two UMMAs, so a third less operand traffic from L2 per flop and half as
 //             many re-reads of the streamed operand from HBM; four stages of 48 KB.  The
-//             epilogue is not overlapped, which is why only the contractions with a long K
-//             (dH: K = V, dW: K = rows of the range) use it.
+//             accumulators do not alternate, so the epilogue is exposed except for what the
+//             half-accumulator order hides: the epilogue drains accumulator 0 first and
+//             releases it, and the UMMA thread starts the next tile with accumulator 0's
+//             share of the first four K-steps while accumulator 1 is still being drained.
+//             dH (K = V) and dW (K = rows of the range) use it with the four epilogue warps;
+//             the single-call logits sweep (short K = d, exp and bf16 stores per element)
+//             uses it with eight epilogue warps, two per TMEM lane quadrant, each taking
+//             half of an accumulator's columns.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -45,7 +51,6 @@ constexpr int kBK = 64;
 constexpr int kABytes = kBM * kBK * 2;     // 16 KB
 constexpr int kBBytes = kHalfN * kBK * 2;  // 16 KB
 constexpr int kOutBytes = kBM * 64 * 2;  // one 128 x 64 bf16 output piece (16 KB), two of them
-constexpr int kGemmThreads = 192;
 constexpr int kTmemCols = 512;
 
 // Shared-memory plan of the two tile shapes.
@@ -57,6 +62,19 @@ struct TileCfg {
   static constexpr int kTileN = NACC * kBN;  // columns of one pair tile
   static constexpr size_t kSmemBytes =
       size_t(kStages) * kStageBytes + kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+// Launch shape of one instantiation.
+template <int MODE, int NACC>
+struct KernelCfg {
+  static constexpr bool kWideSweep = (MODE == 5 /*MODE_LSE_E*/ && NACC == 2);
+  static constexpr int kEpiWarps = kWideSweep ? 8 : 4;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;
+  // bf16 output pieces staged for TMA stores: two per CTA (one per group of four epilogue warps
+  // in the wide sweep, alternating in the 256 x 256 sweeps)
+  static constexpr int kOutTotal = kWideSweep ? 2 * kOutBytes : TileCfg<NACC>::kOutTotal;
+  static constexpr size_t kSmemBytes = size_t(TileCfg<NACC>::kStages) * TileCfg<NACC>::kStageBytes +
+                                       kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
 };
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -111,7 +129,7 @@ __device__ __forceinline__ long long max_ksteps_per_pair(const GemmParams& p, in
   const int npairs = gridDim.x >> 1;
   if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
     if (rows <= 0) return 0;
-    const int VT = (p.V + kBN - 1) / kBN;
+    const int VT = (p.V + kTN - 1) / kTN;
     const int nrb = (rows + kTileM - 1) / kTileM;
     const SweepShape sh = sweep_shape(nrb, p.R, p.C, VT);
     long long tiles = (long long)sh.nfull * ((VT + p.C - 1) / p.C);
@@ -169,7 +187,7 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
   const int pid = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   if (MODE == MODE_LSE || MODE == MODE_GRAD || MODE == MODE_LSE_E) {
     if (rows <= 0) return false;
-    const int VT = (p.V + kBN - 1) / kBN;
+    const int VT = (p.V + kTN - 1) / kTN;
     const int nrb = (rows + kTileM - 1) / kTileM;
     const SweepShape sh = sweep_shape(nrb, p.R, p.C, VT);
     // complete waves: this CTA is (row block rbi, split s) of every wave
@@ -197,7 +215,8 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
       t.split = st;
     }
     t.m0 = row_begin + rbk * kTileM;
-    t.n0 = (vt0 + off) * kBN;
+    t.n0 = (vt0 + off) * kTN;
+    t.nh = (NACC == 2 && t.n0 + kBN < p.V) ? 2 : 1;
     t.ka0 = t.kb0 = 0;
     t.nk = p.d / kBK;
     t.first = (off == 0);
@@ -251,34 +270,41 @@ __device__ __forceinline__ void stage_row_sw128(uint8_t* piece, int r, const uin
 
 // AND-reduction of a predicate over the 128 epilogue threads (named barrier 1), so that
 // the decision to leave the tile loop is taken by all of them together.
+template <int NTHREADS>
 __device__ __forceinline__ bool epilogue_all(bool ok) {
   uint32_t r;
   asm volatile(
       "{\n\t.reg .pred p, q;\n\t"
       "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(r)
-      : "r"((uint32_t)ok)
+      : "r"((uint32_t)ok), "n"(NTHREADS)
       : "memory");
   return r != 0;
 }
+// Named barriers of the eight-warp epilogue: 1 = all 256 threads, 2 + g = the 128 threads of group g.
+__device__ __forceinline__ void epilogue_bar_all256() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_bar_group(int g) {
+  asm volatile("bar.sync %0, 128;" ::"r"(2 + g) : "memory");
+}
 
 template <int MODE, int A_MN, int B_MN, int NACC>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((KernelCfg<MODE, NACC>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-  static_assert(NACC == 1 || (MODE != MODE_LSE && MODE != MODE_GRAD && MODE != MODE_LSE_E),
-                "the vocabulary sweeps need the alternating accumulators of the 256 x 256 tile");
+  static_assert(NACC == 1 || (MODE != MODE_LSE && MODE != MODE_GRAD),
+                "these sweeps are written for the alternating accumulators of the 256 x 256 tile");
   using Cfg = TileCfg<NACC>;
+  using KC = KernelCfg<MODE, NACC>;
   constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // 128-byte swizzle atoms need 1024-byte alignment
   uint8_t* smem = smem_raw + (base - raw);
-  uint8_t* out_smem = smem + kStages * kStageBytes;  // two 16 KB output pieces (NACC = 1 only)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + Cfg::kOutTotal);
-  const uint32_t bar0 = base + kStages * kStageBytes + Cfg::kOutTotal;
+  uint8_t* out_smem = smem + kStages * kStageBytes;  // two 16 KB output pieces (bf16-storing modes)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(out_smem + KC::kOutTotal);
+  const uint32_t bar0 = base + kStages * kStageBytes + KC::kOutTotal;
   // barrier slots: full[kStages], empty[kStages], tmem_full[2], tmem_empty[2].
   // NACC = 1: accumulator b = j & 1 of tile j uses tmem_full[b] / tmem_empty[b].
   // NACC = 2: tmem_full[0] covers both halves of a tile, tmem_empty[h] releases half h.
@@ -318,7 +344,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 8);  // leader's copy is used: 4 epilogue warps of each CTA
+      mbar_init(tempty_bar(b), 2 * KC::kEpiWarps);  // leader's copy is used: the epilogue warps of both CTAs
     }
     *abort_flag = 0;
     mbar_fence_init();
@@ -404,13 +430,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
           d_tmem = tmem_base + buf * kBN;
         } else {
-          // both halves of the previous tile must have been drained
-          if (!mbar_wait(tempty_bar(0), (j & 1u) ^ 1u, abort_flag)) break;
-          if (!mbar_wait(tempty_bar(1), (j & 1u) ^ 1u, abort_flag)) break;
           d_tmem = tmem_base;
         }
-        tc_fence_after();
-        for (int kb = 0; kb < t.nk; ++kb, ++it) {
+        int kb_start = 0;
+        if (NACC == 2) {
+          // Accumulator 0 is released by the epilogue before accumulator 1: start with
+          // accumulator 0's UMMAs of the first `pre` K-steps (their stages are already loaded),
+          // then wait for accumulator 1 and catch up on the same stages.
+          const int pre = t.nk < kStages ? t.nk : kStages;
+          if (!mbar_wait(tempty_bar(0), (j & 1u) ^ 1u, abort_flag)) break;
+          tc_fence_after();
+          for (int kb = 0; ok && kb < pre; ++kb) {
+            const uint32_t itk = it + kb;
+            const int s = itk % kStages;
+            if (!mbar_wait(full_bar(s), (itk / kStages) & 1u, abort_flag)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+#pragma unroll
+            for (int kk = 0; kk < kBK / 16; ++kk) {
+              const uint64_t da = A_MN ? smem_desc_sw128(sa + kk * 2048, 8192, 1024)
+                                       : smem_desc_sw128(sa + kk * 32, 16, 1024);
+              const uint64_t db = B_MN ? smem_desc_sw128(sb + kk * 2048, 8192, 1024)
+                                       : smem_desc_sw128(sb + kk * 32, 16, 1024);
+              umma_bf16(d_tmem, da, db, idesc, (kb | kk) ? 1u : 0u);
+            }
+            if (t.nh == 1) umma_commit_pair(empty_bar(s));
+          }
+          if (!ok) break;
+          if (!mbar_wait(tempty_bar(1), (j & 1u) ^ 1u, abort_flag)) break;
+          tc_fence_after();
+          if (t.nh == 2) {
+            for (int kb = 0; kb < pre; ++kb) {
+              const int s = (it + kb) % kStages;
+              const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes + kBBytes;
+#pragma unroll
+              for (int kk = 0; kk < kBK / 16; ++kk) {
+                const uint64_t da = A_MN ? smem_desc_sw128(sa + kk * 2048, 8192, 1024)
+                                         : smem_desc_sw128(sa + kk * 32, 16, 1024);
+                const uint64_t db = B_MN ? smem_desc_sw128(sb + kk * 2048, 8192, 1024)
+                                         : smem_desc_sw128(sb + kk * 32, 16, 1024);
+                umma_bf16(d_tmem + kBN, da, db, idesc, (kb | kk) ? 1u : 0u);
+              }
+              umma_commit_pair(empty_bar(s));  // both accumulators' UMMAs have read the stage
+            }
+          }
+          it += pre;
+          kb_start = pre;
+        } else {
+          tc_fence_after();
+        }
+        for (int kb = kb_start; kb < t.nk; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag)) {
             ok = false;
@@ -442,7 +514,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     // ------------------------------------------------------------ epilogue warps
     const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32)
     const int r_in_tile = quad * 32 + lane;
-    const bool issuer = (threadIdx.x == 64);  // issues the TMA stores of the bf16 pieces
+    // eight-warp epilogue: warps 2..5 are group 0, warps 6..9 group 1; each group takes half of
+    // an accumulator's columns (four-warp epilogue: one group)
+    const int group = (warp - 2) >> 2;
+    const bool issuer = ((warp - 2) & 3) == 0 && lane == 0;  // issues its group's TMA stores
     // running state of this thread's row across the tiles of a sweep
     float run_m2 = -INFINITY, run_l = 0.f, run_z = 0.f, run_s = 0.f;
     Tile t;
@@ -467,10 +542,113 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
       const bool got = mbar_wait(tfull_bar(buf), (NACC == 1 ? (j >> 1) : j) & 1u, abort_flag);
-      if (!epilogue_all(got)) break;
+      if (!epilogue_all<32 * KC::kEpiWarps>(got)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;
 
+      if (KC::kWideSweep) {
+        // This group's 128 columns of each accumulator, 32 at a time with the next 32 already
+        // on their way from TMEM: exp, sums, bf16; every 64 columns leave through the group's
+        // swizzled piece in shared memory and a TMA store.  An accumulator is handed back to
+        // the UMMA warp as soon as this warp's last load from it has landed.
+        uint8_t* piece = out_smem + group * kOutBytes;
+        const int nchunks = 4 * t.nh;
+        auto chunk_off = [&](int c) { return (c >> 2) * kBN + group * 128 + (c & 3) * 32; };
+        // exp / sums / packing of one 32-column chunk into 16 words of w
+        auto do_chunk = [&](const uint32_t (&r)[32], int c, uint32_t* w16) {
+          const int col0 = t.n0 + chunk_off(c);
+          if (valid && col0 < p.V) {
+            const int ti = tgt - col0;
+            float acc = 0.f, accs = 0.f;
+            if (col0 + 32 <= p.V) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                const float z0 = __uint_as_float(r[i]), z1 = __uint_as_float(r[i + 1]);
+                const float e0 = ex2_approx(fmaf(z0, kLog2e, -ref2));
+                const float e1 = ex2_approx(fmaf(z1, kLog2e, -ref2));
+                acc += e0 + e1;
+                accs = fmaf(e0, z0, fmaf(e1, z1, accs));
+                w16[i >> 1] = pack_bf16x2(e0, e1);
+              }
+            } else {
+              // the vocabulary ends inside these 32 columns: columns past V hold z = 0
+              // (zero-filled W rows) and their e is cleared
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                const float z0 = __uint_as_float(r[i]), z1 = __uint_as_float(r[i + 1]);
+                float e0 = ex2_approx(fmaf(z0, kLog2e, -ref2));
+                float e1 = ex2_approx(fmaf(z1, kLog2e, -ref2));
+                if (col0 + i >= p.V) e0 = 0.f;
+                if (col0 + i + 1 >= p.V) e1 = 0.f;
+                acc += e0 + e1;
+                accs = fmaf(e0, z0, fmaf(e1, z1, accs));
+                w16[i >> 1] = pack_bf16x2(e0, e1);
+              }
+            }
+            run_l += acc;
+            run_s += accs;
+            if (ti >= 0 && ti < 32) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i == ti) run_z = __uint_as_float(r[i]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w16[i] = 0u;
+          }
+        };
+        uint32_t ra[32], rb[32], w[32];
+        tmem_ld32(taddr + chunk_off(0), ra);
+#pragma unroll 1
+        for (int c = 0; c < nchunks; c += 2) {
+          tmem_ld_wait();                                // chunk c is in ra
+          tmem_ld32(taddr + chunk_off(c + 1), rb);
+          do_chunk(ra, c, w);
+          tmem_ld_wait();                                // chunk c + 1 is in rb
+          if (c + 2 < nchunks) tmem_ld32(taddr + chunk_off(c + 2), ra);
+          if (((c + 1) & 3) == 3) {
+            // that was this warp's last load from accumulator (c + 1) / 4
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) >> 2), 0));
+          }
+          do_chunk(rb, c + 1, w + 16);
+          // the group's previous store must have finished reading the piece
+          if (issuer) tma_store_wait_read<0>();
+          epilogue_bar_group(group);
+          stage_row_sw128(piece, r_in_tile, w);
+          fence_proxy_async_smem();
+          epilogue_bar_group(group);
+          if (issuer) {
+            tma_store_2d(&tmC, smem_u32(piece), t.n0 + chunk_off(c), t.m0 - row_begin + (int)rank * kBM);
+            tma_store_commit();
+          }
+        }
+        if (t.nh == 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
+        }
+        if (t.last) {
+          // end of this row block's sweep: group 1 hands its sums to group 0 through its piece
+          float* xch = reinterpret_cast<float*>(out_smem + kOutBytes);
+          if (group == 1) {
+            if (issuer) tma_store_wait_read<0>();
+            epilogue_bar_group(1);
+            xch[r_in_tile * 4 + 0] = run_l;
+            xch[r_in_tile * 4 + 1] = run_z;
+            xch[r_in_tile * 4 + 2] = run_s;
+          }
+          epilogue_bar_all256();
+          if (group == 0 && valid) {
+            const size_t o = (size_t)row * kMaxSplits + t.split;
+            p.pl[o] = run_l + xch[r_in_tile * 4 + 0];
+            p.pz[o] = run_z + xch[r_in_tile * 4 + 1];
+            p.ps[o] = run_s + xch[r_in_tile * 4 + 2];
+          }
+          epilogue_bar_all256();  // group 1 may stage into its piece again
+        }
+        continue;
+      }
       if (MODE == MODE_GRAD || MODE == MODE_LSE_E) {
         // bf16 output tile, 64 columns at a time: registers -> swizzled smem piece -> TMA store
 #pragma unroll 1

@@ -41,7 +41,7 @@ static int env_int(const char* name, int dflt) {
 static bool carve(const oapl_problem* p, int flags, Carve* c) {
   if (!p || p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return false;
   if (p->d % 64 != 0) return false;
-  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000) return false;
+  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 512 > (int64_t)2000000000) return false;
   const size_t n_pad = align_up((size_t)p->N, 256);
   c->n_pad = (int)n_pad;
   c->nblk = (int)((p->N + kScanBlock - 1) / kScanBlock);
@@ -49,7 +49,7 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
   chunk = (int)align_up((size_t)(chunk < 256 ? 256 : chunk), 256);
   if ((size_t)chunk > n_pad) chunk = (int)n_pad;
   c->chunk_rows = chunk;
-  c->ldg = (int)align_up((size_t)p->V, 256);
+  c->ldg = (int)align_up((size_t)p->V, 512);
   size_t off = 0;
   auto take = [&](size_t bytes) {
     const size_t o = off;
@@ -215,7 +215,8 @@ static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtenso
                        const GemmParams& gp, int grid, cudaStream_t st) {
   static bool attr_set = false;
   auto kern = gemm_kernel<MODE, A_MN, B_MN, NACC>;
-  constexpr size_t smem = TileCfg<NACC>::kSmemBytes;
+  constexpr size_t smem = KernelCfg<MODE, NACC>::kSmemBytes;
+  constexpr int threads = KernelCfg<MODE, NACC>::kThreads;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return OAPL_ERR_CUDA;
@@ -225,9 +226,9 @@ static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtenso
   if (slot >= 0 && g_prof_clk_addr) {
     GemmParams timed = gp;
     timed.clk = g_prof_clk_addr + 2 * MODE;
-    kern<<<grid, kGemmThreads, smem, st>>>(a, b, c, timed);
+    kern<<<grid, threads, smem, st>>>(a, b, c, timed);
   } else {
-    kern<<<grid, kGemmThreads, smem, st>>>(a, b, c, gp);
+    kern<<<grid, threads, smem, st>>>(a, b, c, gp);
   }
   OAPL_LAUNCHED();
   prof_end(slot, st);
@@ -238,7 +239,7 @@ static int check_problem(const oapl_problem* p, bool need_loss_inputs) {
   if (!p) return OAPL_ERR_INVALID_ARG;
   if (p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return OAPL_ERR_INVALID_ARG;
   if (p->d % 64 != 0) return OAPL_ERR_UNSUPPORTED_SHAPE;
-  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 256 > (int64_t)2000000000)
+  if (p->N > (int64_t)2000000000 || (int64_t)p->V + 512 > (int64_t)2000000000)
     return OAPL_ERR_UNSUPPORTED_SHAPE;
   if (!p->H || !p->W || !p->targets || !p->mask || !p->seq_id) return OAPL_ERR_INVALID_ARG;
   if (((uintptr_t)p->H | (uintptr_t)p->W) & 15) return OAPL_ERR_MISALIGNED;
@@ -391,7 +392,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   float* ztc = reinterpret_cast<float*>(w + c.ztc);
   float* rowscale = reinterpret_cast<float*>(w + c.rowscale);
   RangeRec* ranges = reinterpret_cast<RangeRec*>(w + c.ranges);
-  const int vtiles = (p->V + kBN - 1) / kBN;
+  const int vtiles = (p->V + 2 * kBN - 1) / (2 * kBN);  // the single-call sweep walks 512-column tiles
 
   CK(cudaMemsetAsync(seq_D, 0, 4 * (size_t)p->S, st));
   if (seq_logp) CK(cudaMemsetAsync(seq_logp, 0, 4 * (size_t)p->S, st));
@@ -450,7 +451,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
     set_lockstep(&gp, w, c, 3 * k, p->d / kBK);
-    rc = launch_gemm<MODE_LSE_E, 0, 0>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
+    rc = launch_gemm<MODE_LSE_E, 0, 0, 2>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
     merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
                                          reinterpret_cast<float*>(w + c.ent_c), alpha, ztc, token_logp, state);
