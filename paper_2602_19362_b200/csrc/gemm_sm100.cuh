@@ -68,11 +68,14 @@ struct TileCfg {
 template <int MODE, int NACC>
 struct KernelCfg {
   static constexpr bool kWideSweep = (MODE == 5 /*MODE_LSE_E*/ && NACC == 2);
+  static constexpr bool kReduceOut = (MODE == 3 /*MODE_DW*/ && NACC == 2);  // fp32 tile added by TMA
   static constexpr int kEpiWarps = kWideSweep ? 8 : 4;
   static constexpr int kThreads = 64 + 32 * kEpiWarps;
-  // bf16 output pieces staged for TMA stores: two per CTA (one per group of four epilogue warps
-  // in the wide sweep, alternating in the 256 x 256 sweeps)
-  static constexpr int kOutTotal = kWideSweep ? 2 * kOutBytes : TileCfg<NACC>::kOutTotal;
+  // bf16 output pieces staged for TMA stores: two alternating 128 x 64 pieces in the 256 x 256
+  // sweeps; two alternating 128 x 32 pieces for each group of four epilogue warps in the wide one
+  // the dW tiles: two alternating 128 x 32 fp32 pieces
+  static constexpr int kOutTotal =
+      kWideSweep ? 4 * (kOutBytes / 2) : (kReduceOut ? 2 * kOutBytes : TileCfg<NACC>::kOutTotal);
   static constexpr size_t kSmemBytes = size_t(TileCfg<NACC>::kStages) * TileCfg<NACC>::kStageBytes +
                                        kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
 };
@@ -258,6 +261,10 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
   }
 }
 
+// Column offset, inside a 256 x 512 tile, of 32-column chunk c of epilogue group g: the group's
+// 128 columns of accumulator c / 4.
+__device__ __forceinline__ int chunk_off_of(int c, int g) { return (c >> 2) * 256 + g * 128 + (c & 3) * 32; }
+
 // Write one thread's 64 bf16 values (32 packed words) as row r of a 128 x 64 piece in the
 // 128-byte-swizzled layout the TMA store expects (16-byte chunk j of row r sits at chunk
 // j ^ (r & 7)); consecutive rows hit different banks.
@@ -266,6 +273,15 @@ __device__ __forceinline__ void stage_row_sw128(uint8_t* piece, int r, const uin
 #pragma unroll
   for (int jc = 0; jc < 8; ++jc)
     rowp[jc ^ (r & 7)] = make_uint4(w[4 * jc], w[4 * jc + 1], w[4 * jc + 2], w[4 * jc + 3]);
+}
+
+// The same for 32 bf16 values (16 words) as row r of a 128 x 32 piece in the 64-byte-swizzled
+// layout (16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)).
+__device__ __forceinline__ void stage_row_sw64(uint8_t* piece, int r, const uint32_t* w) {
+  uint4* rowp = reinterpret_cast<uint4*>(piece + r * 64);
+#pragma unroll
+  for (int jc = 0; jc < 4; ++jc)
+    rowp[jc ^ ((r >> 1) & 3)] = make_uint4(w[4 * jc], w[4 * jc + 1], w[4 * jc + 2], w[4 * jc + 3]);
 }
 
 // AND-reduction of a predicate over the 128 epilogue threads (named barrier 1), so that
@@ -548,12 +564,27 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 
       if (KC::kWideSweep) {
         // This group's 128 columns of each accumulator, 32 at a time with the next 32 already
-        // on their way from TMEM: exp, sums, bf16; every 64 columns leave through the group's
-        // swizzled piece in shared memory and a TMA store.  An accumulator is handed back to
-        // the UMMA warp as soon as this warp's last load from it has landed.
-        uint8_t* piece = out_smem + group * kOutBytes;
+        // on their way from TMEM: exp, sums, bf16; each 32 columns leave through one of the
+        // group's two swizzled pieces in shared memory and a TMA store (tmC has 128 x 32
+        // boxes).  An accumulator is handed back to the UMMA warp as soon as this warp's last
+        // load from it has landed.
+        constexpr int kPiece = kOutBytes / 2;
         const int nchunks = 4 * t.nh;
-        auto chunk_off = [&](int c) { return (c >> 2) * kBN + group * 128 + (c & 3) * 32; };
+        // stage 32 columns and send them off; the store two pieces back has drained the buffer
+        auto send_chunk = [&](int c, const uint32_t* w16) {
+          uint8_t* piece = out_smem + (group * 2 + (c & 1)) * kPiece;
+          if (issuer) tma_store_wait_read<1>();
+          epilogue_bar_group(group);
+          stage_row_sw64(piece, r_in_tile, w16);
+          fence_proxy_async_smem();
+          epilogue_bar_group(group);
+          if (issuer) {
+            tma_store_2d(&tmC, smem_u32(piece), t.n0 + chunk_off_of(c, group),
+                         t.m0 - row_begin + (int)rank * kBM);
+            tma_store_commit();
+          }
+        };
+        auto chunk_off = [&](int c) { return chunk_off_of(c, group); };
         // exp / sums / packing of one 32-column chunk into 16 words of w
         auto do_chunk = [&](const uint32_t (&r)[32], int c, uint32_t* w16) {
           const int col0 = t.n0 + chunk_off(c);
@@ -597,13 +628,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int i = 0; i < 16; ++i) w16[i] = 0u;
           }
         };
-        uint32_t ra[32], rb[32], w[32];
+        uint32_t ra[32], rb[32], w[16];
         tmem_ld32(taddr + chunk_off(0), ra);
 #pragma unroll 1
         for (int c = 0; c < nchunks; c += 2) {
           tmem_ld_wait();                                // chunk c is in ra
           tmem_ld32(taddr + chunk_off(c + 1), rb);
           do_chunk(ra, c, w);
+          send_chunk(c, w);
           tmem_ld_wait();                                // chunk c + 1 is in rb
           if (c + 2 < nchunks) tmem_ld32(taddr + chunk_off(c + 2), ra);
           if (((c + 1) & 3) == 3) {
@@ -612,17 +644,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) >> 2), 0));
           }
-          do_chunk(rb, c + 1, w + 16);
-          // the group's previous store must have finished reading the piece
-          if (issuer) tma_store_wait_read<0>();
-          epilogue_bar_group(group);
-          stage_row_sw128(piece, r_in_tile, w);
-          fence_proxy_async_smem();
-          epilogue_bar_group(group);
-          if (issuer) {
-            tma_store_2d(&tmC, smem_u32(piece), t.n0 + chunk_off(c), t.m0 - row_begin + (int)rank * kBM);
-            tma_store_commit();
-          }
+          do_chunk(rb, c + 1, w);
+          send_chunk(c + 1, w);
         }
         if (t.nh == 1) {
           __syncwarp();
@@ -630,7 +653,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         if (t.last) {
           // end of this row block's sweep: group 1 hands its sums to group 0 through its piece
-          float* xch = reinterpret_cast<float*>(out_smem + kOutBytes);
+          float* xch = reinterpret_cast<float*>(out_smem + 2 * kPiece);
           if (group == 1) {
             if (issuer) tma_store_wait_read<0>();
             epilogue_bar_group(1);
@@ -646,6 +669,50 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             p.ps[o] = run_s + xch[r_in_tile * 4 + 2];
           }
           epilogue_bar_all256();  // group 1 may stage into its piece again
+        }
+        continue;
+      }
+      if (KC::kReduceOut) {
+        // dW += tile: 32 fp32 columns at a time through one of two swizzled 128 x 32 pieces in
+        // shared memory and a TMA reduce-add (tmC maps dW), so the old values never travel to
+        // the SM.  Every element of dW belongs to one tile of the launch and launches follow
+        // one another on the stream, so the sums are formed in a fixed order.  Rows past V and
+        // columns past d are clipped by the tensor map.
+        const int nchunks = t.nh * (kBN / 32);
+        uint32_t ra[32], rb[32];
+        auto send32 = [&](int c, const uint32_t (&r)[32]) {
+          uint8_t* piece = out_smem + (c & 1) * kOutBytes;
+          if (issuer) tma_store_wait_read<1>();
+          epilogue_bar_sync();
+          stage_row_sw128(piece, r_in_tile, r);
+          fence_proxy_async_smem();
+          epilogue_bar_sync();
+          if (issuer) {
+            if (t.n0 + c * 32 < p.d && t.m0 + (int)rank * kBM < p.V)  // box not wholly outside
+              tma_reduce_add_2d(&tmC, smem_u32(piece), t.n0 + c * 32, t.m0 + (int)rank * kBM);
+            // one group per piece, also when it is empty: the wait above counts groups
+            tma_store_commit();
+          }
+        };
+        tmem_ld32(taddr, ra);
+#pragma unroll 1
+        for (int c = 0; c < nchunks; c += 2) {
+          tmem_ld_wait();
+          tmem_ld32(taddr + (c + 1) * 32, rb);
+          send32(c, ra);
+          tmem_ld_wait();
+          if (c + 2 < nchunks) tmem_ld32(taddr + (c + 2) * 32, ra);
+          if (c + 1 == kBN / 32 - 1 || c + 1 == 2 * (kBN / 32) - 1) {
+            // this warp's last load from accumulator (c + 1) / 8 has landed
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) / (kBN / 32)), 0));
+          }
+          send32(c + 1, rb);
+        }
+        if (t.nh == 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
         }
         continue;
       }
@@ -818,7 +885,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
     }
-    if (issuer && (MODE == MODE_GRAD || MODE == MODE_LSE_E)) tma_store_wait_all();
+    if (issuer && (MODE == MODE_GRAD || MODE == MODE_LSE_E || KC::kReduceOut)) tma_store_wait_all();
   }
 
   // ---------------------------------------------------------------- teardown

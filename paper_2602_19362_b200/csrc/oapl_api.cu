@@ -140,6 +140,34 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t c
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen through 128-row x 32-column boxes (64-byte rows, 64-byte swizzle): the
+// store map of the wide logits sweep.
+static bool make_map_store32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 matrix [rows, cols] row-major seen through 128-row x 32-column boxes (128-byte rows,
+// 128-byte swizzle): the reduce-add map of the dW contraction.
+static bool make_map_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 4};
+  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 static int sm_count() {
   static int n = 0;
   if (!n) {
@@ -416,14 +444,16 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, c.max_ranges, ranges, state);
   CKL();
 
-  CUtensorMap tmH, tmW, tmEk, tmWmn, tmEmn, tmHsmn;
+  CUtensorMap tmH, tmW, tmEk, tmEst, tmWmn, tmEmn, tmHsmn, tmdW;
   const uint64_t ldg = (uint64_t)c.ldg;
   bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmEk, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 128) &&
+            make_map_store32(&tmEst, E, (uint64_t)c.stage_alloc_rows, ldg, ldg) &&
             make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
             make_map(&tmEmn, E, (uint64_t)c.stage_alloc_rows, ldg, ldg, 64) &&
-            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 256, (uint64_t)p->d, (uint64_t)p->d, 64);
+            make_map(&tmHsmn, Hs, (uint64_t)c.n_pad + 256, (uint64_t)p->d, (uint64_t)p->d, 64) &&
+            make_map_f32(&tmdW, dW, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d);
   if (!ok) return OAPL_ERR_CUDA;
 
   GemmParams gp;
@@ -451,7 +481,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
     set_lockstep(&gp, w, c, 3 * k, p->d / kBK);
-    rc = launch_gemm<MODE_LSE_E, 0, 0, 2>(tmH, tmW, tmEk, gp, 2 * gp.R * gp.C, st);
+    rc = launch_gemm<MODE_LSE_E, 0, 0, 2>(tmH, tmW, tmEst, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
     merge_e_kernel<<<n_sm, 256, 0, st>>>(gp.pl, gp.pz, gp.ps, zref, rg, gp.R, gp.C, vtiles, live_rows, lse, lp_c,
                                          reinterpret_cast<float*>(w + c.ent_c), alpha, ztc, token_logp, state);
@@ -471,7 +501,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
                                                  lse, ztc, rg, p->d, p->V, c.ldg, Hs, rowscale, E);
     CKL();
     set_lockstep(&gp, w, c, 3 * k + 1, 0);
-    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmEmn, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmdW, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
     gp.rowscale = rowscale;
     set_lockstep(&gp, w, c, 3 * k + 2, 0);
@@ -609,14 +639,15 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   CKL();
   if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
 
-  CUtensorMap tmH, tmW, tmGk, tmWmn, tmGmn, tmHmn;
+  CUtensorMap tmH, tmW, tmGk, tmWmn, tmGmn, tmHmn, tmdW;
   const uint64_t ldg = (uint64_t)c.ldg;
   bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmGk, G, (uint64_t)c.chunk_rows, ldg, ldg, 128) &&
             make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
             make_map(&tmGmn, G, (uint64_t)c.chunk_rows, ldg, ldg, 64) &&
-            make_map(&tmHmn, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 64);
+            make_map(&tmHmn, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 64) &&
+            make_map_f32(&tmdW, dW, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d);
   if (!ok) return OAPL_ERR_CUDA;
 
   GemmParams gp;
@@ -652,7 +683,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
     rc = launch_gemm<MODE_DH, 0, 1, 2>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
     set_lockstep(&gp, w, c, slot++, 0);
-    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmGmn, tmHmn, tmGmn, gp, n_sm & ~1, st);
+    rc = launch_gemm<MODE_DW, 1, 1, 2>(tmGmn, tmHmn, tmdW, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
   }
   return OAPL_OK;
