@@ -570,13 +570,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // load from it has landed.
         constexpr int kPiece = kOutBytes / 2;
         const int nchunks = 4 * t.nh;
-        // stage 32 columns and send them off; the store two pieces back has drained the buffer
+        // Stage 32 columns and send them off.  One barrier per piece: before it the issuing
+        // thread has seen every earlier store finish reading shared memory, so whoever passes
+        // it may overwrite the other buffer (last read by the previous piece's store) next time.
         auto send_chunk = [&](int c, const uint32_t* w16) {
           uint8_t* piece = out_smem + (group * 2 + (c & 1)) * kPiece;
-          if (issuer) tma_store_wait_read<1>();
-          epilogue_bar_group(group);
           stage_row_sw64(piece, r_in_tile, w16);
           fence_proxy_async_smem();
+          if (issuer) tma_store_wait_read<0>();
           epilogue_bar_group(group);
           if (issuer) {
             tma_store_2d(&tmC, smem_u32(piece), t.n0 + chunk_off_of(c, group),
@@ -680,17 +681,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // columns past d are clipped by the tensor map.
         const int nchunks = t.nh * (kBN / 32);
         uint32_t ra[32], rb[32];
+        // one barrier per piece: before it the issuing thread has seen every earlier reduce
+        // finish reading shared memory, so the other buffer may be overwritten next time
         auto send32 = [&](int c, const uint32_t (&r)[32]) {
           uint8_t* piece = out_smem + (c & 1) * kOutBytes;
-          if (issuer) tma_store_wait_read<1>();
-          epilogue_bar_sync();
           stage_row_sw128(piece, r_in_tile, r);
           fence_proxy_async_smem();
+          if (issuer) tma_store_wait_read<0>();
           epilogue_bar_sync();
           if (issuer) {
             if (t.n0 + c * 32 < p.d && t.m0 + (int)rank * kBM < p.V)  // box not wholly outside
               tma_reduce_add_2d(&tmC, smem_u32(piece), t.n0 + c * 32, t.m0 + (int)rank * kBM);
-            // one group per piece, also when it is empty: the wait above counts groups
             tma_store_commit();
           }
         };
