@@ -229,13 +229,13 @@ def run_cuda(args) -> None:
         B.oapl_group_advantage(batch["reward"], batch["group_id"], P, 1e-6, adv)
         clip_frac = torch.zeros(1, device=dev)
 
-    def step():
-        local_step()
+    def step(prob=prob, loss=loss, seq_logp=seq_logp, dH=dH, dW=dW):
+        local_step(prob, loss, seq_logp, dH, dW)
         if world > 1:
             # the one exchange of the data-parallel step: sum of dW (and of the loss) over the ranks
             dp.allreduce_outputs(loss, dW)
 
-    def local_step():
+    def local_step(prob, loss, seq_logp, dH, dW):
         if grpo:
             B.oapl_grpo_loss_fwd_bwd(prob, logp_old, adv, 0.2, loss, seq_logp, None, clip_frac, dH, dW, False, ws)
         elif fused:
@@ -314,7 +314,11 @@ def run_cuda(args) -> None:
                               "peak_kind": f"hbm_gbs of {measured_peaks()['source']}"}}
         del Wopt, master, m_st, v_st
 
-    # ---- end to end: host-resident inputs and results, copies inside the timed region
+    # ---- end to end: host-resident inputs and results, copies inside the timed region.
+    # Every step copies its inputs from pinned host memory and its results (loss, sequence
+    # log-probs, dH, dW) back.  The caller pipelines the steps the way a trainer would: two sets
+    # of device buffers, one copy-in stream, the compute stream, one copy-out stream, so that the
+    # copies of step k+1 and k-1 run under the kernels of step k.
     e2e = None
     if not args.no_e2e:
         names = ["H", "targets", "mask", "seq_id", "group_id", "reward", "logp_inf"]
@@ -322,29 +326,58 @@ def run_cuda(args) -> None:
         host_out = {"loss": torch.empty(1).pin_memory(), "seq_logp": torch.empty(S).pin_memory(),
                     "dH": torch.empty(N, d, dtype=torch.bfloat16).pin_memory(),
                     "dW": torch.empty(V, d, dtype=torch.float32).pin_memory()}
-        dev_out = {"loss": loss, "seq_logp": seq_logp, "dH": dH, "dW": dW}
         h2d = sum(t.numel() * t.element_size() for t in host_in.values())
         d2h = sum(t.numel() * t.element_size() for t in host_out.values())
+        slots = []
+        for i in range(2):
+            b_i = batch if i == 0 else {k: (v.clone() if (torch.is_tensor(v) and k in names) else v)
+                                        for k, v in batch.items()}
+            o_i = {"loss": loss, "seq_logp": seq_logp, "dH": dH, "dW": dW} if i == 0 else \
+                  {"loss": torch.zeros_like(loss), "seq_logp": torch.zeros_like(seq_logp),
+                   "dH": torch.empty_like(dH), "dW": torch.empty_like(dW)}
+            slots.append({"batch": b_i, "prob": B.make_problem(b_i, loss_scale=1.0 / (S * world)), "out": o_i,
+                          "in_done": torch.cuda.Event(), "comp_done": torch.cuda.Event(),
+                          "out_done": torch.cuda.Event()})
+        s_in, s_out, s_comp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
 
-        def e2e_step():
-            for k in names:
-                batch[k].copy_(host_in[k], non_blocking=True)
-            step()
-            for k, t in host_out.items():
-                t.copy_(dev_out[k], non_blocking=True)
+        def e2e_steps(n):
+            for k in range(n):
+                sl = slots[k & 1]
+                with torch.cuda.stream(s_in):
+                    if k >= 2:
+                        s_in.wait_event(sl["comp_done"])      # the step that read this input set is done
+                    for name in names:
+                        sl["batch"][name].copy_(host_in[name], non_blocking=True)
+                    sl["in_done"].record(s_in)
+                s_comp.wait_event(sl["in_done"])
+                if k >= 2:
+                    s_comp.wait_event(sl["out_done"])         # this output set has been copied out
+                step(sl["prob"], sl["out"]["loss"], sl["out"]["seq_logp"], sl["out"]["dH"], sl["out"]["dW"])
+                sl["comp_done"].record(s_comp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(sl["comp_done"])
+                    for name, t in host_out.items():
+                        t.copy_(sl["out"][name], non_blocking=True)
+                    sl["out_done"].record(s_out)
+            for sl in slots[:min(n, 2)]:
+                s_comp.wait_event(sl["out_done"])
 
-        e2e_step()
+        e2e_steps(2)
         barrier()
-        n_e2e = max(1, min(args.steps, 3))
+        n_e2e = max(4, args.steps)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(n_e2e):
-            e2e_step()
+        e2e_steps(n_e2e)
         e1.record()
         barrier()
         e2e_ms = reduce_max(e0.elapsed_time(e1) / n_e2e, dist if world > 1 else None, dev)
         e2e = {"value": tokens_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e}
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e,
+               "pipelining": "two device buffer sets; copy-in, compute and copy-out streams"}
+        st = B.oapl_get_last_status(ws)
+        if st != 0:
+            raise RuntimeError(f"device status {B.STATUS.get(st, st)} in the end-to-end loop")
+        del slots
 
     if rank != 0:
         if world > 1:

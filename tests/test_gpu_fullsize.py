@@ -13,11 +13,12 @@ from tests import helpers as hp
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,fused,beta", [("7b", True, 1.0), ("7b", False, 1.0), ("14b-long", True, 1.0),
-                                             ("lag-stress", True, 0.1)],
-                         ids=["7b-single-call", "7b-two-calls", "14b-long-single-call", "lag-stress-single-call"])
+@pytest.mark.parametrize("name,fused,beta", [("7b", True, 1.0), ("7b", False, 1.0), ("1.5b", True, 1.0),
+                                             ("14b-long", True, 1.0), ("lag-stress", True, 0.1)],
+                         ids=["7b-single-call", "7b-two-calls", "1.5b-single-call", "14b-long-single-call",
+                              "lag-stress-single-call"])
 def test_full_size_sampled_rows_and_invariants(name, fused, beta):
-    # 14b-long: packed rows, sequences of up to 16384 tokens, d = 5120; lag-stress: 2.5 M response
+    # 1.5b: V = 151936 ends inside a 512-column tile; 14b-long: packed rows, sequences of up to 16384 tokens, d = 5120; lag-stress: 2.5 M response
     # tokens, logits scaled by 4 (peaked distributions), 25 % of the groups without any reward
     wl = synth.WORKLOADS[name]
     dev = synth.make_batch(wl, seed=0, device="cuda", beta=beta)
