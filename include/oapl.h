@@ -41,7 +41,10 @@ typedef enum {
   OAPL_ERR_DEVICE_TIMEOUT = -8,      /* device: a bounded pipeline wait expired */
   OAPL_ERR_CUDA = -9,                /* a CUDA runtime/driver call failed */
   OAPL_ERR_BAD_STATE = -10,          /* oapl_loss_bwd without a matching oapl_loss_fwd in ws */
-  OAPL_ERR_SEQUENCE_TOO_LONG = -11   /* device: oapl_loss_fwd_bwd met a sequence longer than its staging capacity */
+  OAPL_ERR_SEQUENCE_TOO_LONG = -11,  /* device: oapl_loss_fwd_bwd met a sequence longer than its staging capacity */
+  OAPL_ERR_OUT_OF_RANGE = -12        /* device: a row's staged exponentials overflowed or vanished (single-call
+                                        paths: some logit exceeds the target's by more than ~128, or H / W hold
+                                        non-finite values); use oapl_loss_fwd + oapl_loss_bwd for such inputs */
 } oapl_status;
 
 /* flags */
@@ -135,7 +138,8 @@ int oapl_loss_bwd(const oapl_problem* problem /*host*/, void* dH, float* dW, int
  * it does not grow with N*V; a sequence with more live rows than that cannot be staged and
  * raises OAPL_ERR_SEQUENCE_TOO_LONG in the status word (outputs are then not meaningful;
  * use the two separate calls).  A target whose probability under the policy is below
- * e^-128 is outside the range of the staged exponentials.
+ * about e^-128 is outside the range of the staged exponentials: the row's sum overflows and
+ * the status word becomes OAPL_ERR_OUT_OF_RANGE.
  */
 int oapl_loss_fwd_bwd(const oapl_problem* problem /*host*/, float* loss, float* seq_logp, float* vhat,
                       float* delta /*may be NULL*/, float* token_logp /*may be NULL*/, void* dH, float* dW,

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "liboapl.so")
 OAPL_OK = 0
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL",
           -4: "UNSUPPORTED_SHAPE", -5: "BAD_TARGET", -6: "BAD_SEQ_ORDER", -7: "NONFINITE_INPUT",
-          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE", -11: "SEQUENCE_TOO_LONG"}
+          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE", -11: "SEQUENCE_TOO_LONG", -12: "OUT_OF_RANGE"}
 OAPL_FLAG_FUSED = 1
 
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",

@@ -544,6 +544,7 @@ const char* oapl_status_string(int status) {
     case OAPL_ERR_CUDA: return "CUDA call failed";
     case OAPL_ERR_BAD_STATE: return "backward called without a matching forward";
     case OAPL_ERR_SEQUENCE_TOO_LONG: return "a sequence has more live rows than the staging capacity";
+    case OAPL_ERR_OUT_OF_RANGE: return "staged exponentials out of range (logit far above the target's, or non-finite input)";
     default: return "unknown status";
   }
 }

@@ -397,6 +397,9 @@ __global__ void merge_e_kernel(const float* __restrict__ pl, const float* __rest
       sz += ps[o + s];
       z += pz[o + s];
     }
+    // the per-row reference is the target logit + 40: a sum that is not a positive finite
+    // number means some logit was more than ~128 above the target's (or the inputs are not finite)
+    if (!(L > 0.f) || !isfinite(L)) set_error(&st->status, -12);
     const float l = zref[i] + logf(L);
     lse[i] = l;
     ent_c[i] = l - sz / L;

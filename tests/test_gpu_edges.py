@@ -125,3 +125,25 @@ def test_device_detected_input_errors_are_reported_not_trapped():
     # the context is still usable afterwards
     good = hp.run_gpu(hp.to_dev(base))
     assert good["status"] == 0
+
+
+def test_single_call_reports_a_target_far_below_the_largest_logit():
+    # one row whose target logit is ~190 below the largest one: exp(z - z_target - 40) overflows
+    # fp32; the single call must say so, the two-call path (online maximum) still matches the oracle
+    wl = dataclasses.replace(TINY, d=64, V=512)
+    cpu = synth.make_batch(wl, seed=10)
+    row = int(torch.nonzero(cpu["mask"])[3])
+    cpu["W"][5] = 0.0
+    cpu["W"][5, 0] = 16.0
+    cpu["W"][9] = 0.0
+    cpu["W"][9, 0] = -8.0
+    cpu["H"][row] = 0.0
+    cpu["H"][row, 0] = 8.0                       # z[5] = 128, z[9] = -64, the others 0
+    cpu["targets"][row] = 9
+    cpu["logp_inf"][row] = -192.0
+    assert hp.run_gpu(hp.to_dev(cpu), fused=True)["status"] == -12
+    out = hp.run_gpu(hp.to_dev(cpu))
+    ref = hp.run_oracle(cpu)
+    assert out["status"] == 0
+    assert abs(float(out["token_logp"][row]) - ref["token_logp"][row]) <= hp.TOL_TOKEN
+    hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
