@@ -383,6 +383,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // the leader CTA's producer keeps the pair in step with the other pairs (its partner
       // follows through the shared pipeline barriers)
       bool meet = p.sync_ctr != nullptr && p.sync_every > 0 && rank == 0;
+      const uint64_t pol_keep = l2_policy_evict_last();
       const unsigned int npairs = gridDim.x >> 1;
       unsigned int epochs = 0;
       for (int j = 0; ok && get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
@@ -405,6 +406,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (A_MN) {
 #pragma unroll
             for (int b = 0; b < kBM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, fb, am + 64 * b, ka);
+          } else if (KC::kWideSweep) {
+            // the pair's H block is read again for every vocabulary tile: keep it in L2
+            tma_load_2d_hint(sa, &tmA, fb, ka, am, pol_keep);
           } else {
             tma_load_2d(sa, &tmA, fb, ka, am);
           }
@@ -569,6 +573,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // boxes).  An accumulator is handed back to the UMMA warp as soon as this warp's last
         // load from it has landed.
         constexpr int kPiece = kOutBytes / 2;
+        const uint64_t pol_stream = l2_policy_evict_first();
         const int nchunks = 4 * t.nh;
         // Stage 32 columns and send them off.  One barrier per piece: before it the issuing
         // thread has seen every earlier store finish reading shared memory, so whoever passes
@@ -580,8 +585,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (issuer) tma_store_wait_read<0>();
           epilogue_bar_group(group);
           if (issuer) {
-            tma_store_2d(&tmC, smem_u32(piece), t.n0 + chunk_off_of(c, group),
-                         t.m0 - row_begin + (int)rank * kBM);
+            // the staged exponentials are not read again before the whole range is written
+            tma_store_2d_hint(&tmC, smem_u32(piece), t.n0 + chunk_off_of(c, group),
+                              t.m0 - row_begin + (int)rank * kBM, pol_stream);
             tma_store_commit();
           }
         };
