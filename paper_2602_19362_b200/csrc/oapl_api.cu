@@ -19,7 +19,9 @@ namespace oapl {
 static std::atomic<uint64_t> g_launches{0};
 #define OAPL_LAUNCHED() (g_launches.fetch_add(1, std::memory_order_relaxed))
 
-constexpr int kChunkRowsDefault = 74 * 128;  // half of a 148-SM wave of row blocks
+// rows of one g chunk of the two-call backward: 74 row blocks of 256, so that on 74 CTA pairs the
+// chunk's dH tiles (74 x d/512) fill whole rounds and its sweep two whole waves of 37 row blocks
+constexpr int kChunkRowsDefault = 74 * 256;
 constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref) in the single-call path
 constexpr int kSyncSlots = 4096;             // lock-step counters in the workspace, one per contraction launch
 

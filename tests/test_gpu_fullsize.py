@@ -30,7 +30,7 @@ def test_full_size_sampled_rows_and_invariants(name, fused, beta):
     # --- sampled live rows (first, last, tile and chunk boundaries, random): token log-prob and dH row
     live = torch.nonzero(mask).flatten()
     g = torch.Generator().manual_seed(0)
-    pick = torch.cat([torch.tensor([0, 1, 127, 128, 9471, 9472, live.numel() - 1]),
+    pick = torch.cat([torch.tensor([0, 1, 127, 128, 9471, 9472, 18943, 18944, live.numel() - 1]),
                       torch.randint(0, live.numel(), (41,), generator=g)])
     rows = live[pick.to(live.device)]
     Wd = orc.bf16_bits_to_f64(synth.bf16_bits(dev["W"]))
