@@ -68,14 +68,16 @@ struct TileCfg {
 template <int MODE, int NACC>
 struct KernelCfg {
   static constexpr bool kWideSweep = (MODE == 5 /*MODE_LSE_E*/ && NACC == 2);
+  static constexpr bool kWideLse = (MODE == 0 /*MODE_LSE*/ && NACC == 2);  // online log-sum-exp, no output tile
   static constexpr bool kReduceOut = (MODE == 3 /*MODE_DW*/ && NACC == 2);  // fp32 tile added by TMA
-  static constexpr int kEpiWarps = kWideSweep ? 8 : 4;
+  static constexpr int kEpiWarps = (kWideSweep || kWideLse) ? 8 : 4;
   static constexpr int kThreads = 64 + 32 * kEpiWarps;
   // bf16 output pieces staged for TMA stores: two alternating 128 x 64 pieces in the 256 x 256
   // sweeps; two alternating 128 x 32 pieces for each group of four epilogue warps in the wide one
   // the dW tiles: two alternating 128 x 32 fp32 pieces
   static constexpr int kOutTotal =
-      kWideSweep ? 4 * (kOutBytes / 2) : (kReduceOut ? 2 * kOutBytes : TileCfg<NACC>::kOutTotal);
+      kWideSweep ? 4 * (kOutBytes / 2)
+                 : (kReduceOut ? 2 * kOutBytes : (kWideLse ? 2048 /*sums of one group*/ : TileCfg<NACC>::kOutTotal));
   static constexpr size_t kSmemBytes = size_t(TileCfg<NACC>::kStages) * TileCfg<NACC>::kStageBytes +
                                        kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
 };
@@ -309,8 +311,8 @@ template <int MODE, int A_MN, int B_MN, int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((KernelCfg<MODE, NACC>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-  static_assert(NACC == 1 || (MODE != MODE_LSE && MODE != MODE_GRAD),
-                "these sweeps are written for the alternating accumulators of the 256 x 256 tile");
+  static_assert(NACC == 1 || MODE != MODE_GRAD,
+                "this sweep is written for the alternating accumulators of the 256 x 256 tile");
   using Cfg = TileCfg<NACC>;
   using KC = KernelCfg<MODE, NACC>;
   constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
@@ -406,7 +408,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (A_MN) {
 #pragma unroll
             for (int b = 0; b < kBM / 64; ++b) tma_load_2d(sa + b * 8192, &tmA, fb, am + 64 * b, ka);
-          } else if (KC::kWideSweep) {
+          } else if (KC::kWideSweep || KC::kWideLse) {
             // the pair's H block is read again for every vocabulary tile: keep it in L2
             tma_load_2d_hint(sa, &tmA, fb, ka, am, pol_keep);
           } else {
@@ -566,6 +568,89 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;
 
+      if (KC::kWideLse) {
+        // Online log-sum-exp over this group's 128 columns of each accumulator, 32 at a time with
+        // the next 32 already on their way from TMEM; nothing is stored per element.
+        const int nchunks = 4 * t.nh;
+        auto lse_chunk = [&](const uint32_t (&r)[32], int c) {
+          const int col0 = t.n0 + chunk_off_of(c, group);
+          if (!valid || col0 >= p.V) return;
+          float v[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+          if (col0 + 32 > p.V) {
+            // a large finite negative: its exponential is 0 and 0 * v stays 0 (no NaN)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i >= p.V) v[i] = -3.0e38f;
+          }
+          float cmax = v[0];
+#pragma unroll
+          for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+          const float m2 = fmaxf(run_m2, cmax * kLog2e);
+          float acc = 0.f, accs = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float e = ex2_approx(fmaf(v[i], kLog2e, -m2));
+            acc += e;
+            accs = fmaf(e, v[i], accs);
+          }
+          const float resc = ex2_approx(run_m2 - m2);
+          run_l = run_l * resc + acc;
+          run_s = run_s * resc + accs;
+          run_m2 = m2;
+          const int ti = tgt - col0;
+          if (ti >= 0 && ti < 32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (i == ti) run_z = v[i];
+          }
+        };
+        uint32_t ra[32], rb[32];
+        tmem_ld32(taddr + chunk_off_of(0, group), ra);
+#pragma unroll 1
+        for (int c = 0; c < nchunks; c += 2) {
+          tmem_ld_wait();
+          tmem_ld32(taddr + chunk_off_of(c + 1, group), rb);
+          lse_chunk(ra, c);
+          tmem_ld_wait();
+          if (c + 2 < nchunks) tmem_ld32(taddr + chunk_off_of(c + 2, group), ra);
+          if (((c + 1) & 3) == 3) {
+            // that was this warp's last load from accumulator (c + 1) / 4
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) >> 2), 0));
+          }
+          lse_chunk(rb, c + 1);
+        }
+        if (t.nh == 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
+        }
+        if (t.last) {
+          // end of this row block's sweep: merge the two groups' (max, sum-exp, sum exp*z, target logit)
+          float* xch = reinterpret_cast<float*>(out_smem);
+          if (group == 1) {
+            xch[r_in_tile * 4 + 0] = run_m2;
+            xch[r_in_tile * 4 + 1] = run_l;
+            xch[r_in_tile * 4 + 2] = run_s;
+            xch[r_in_tile * 4 + 3] = run_z;
+          }
+          epilogue_bar_all256();
+          if (group == 0 && valid) {
+            const float m1 = xch[r_in_tile * 4 + 0];
+            const float M = fmaxf(run_m2, m1);
+            const float w0 = ex2_approx(run_m2 - M), w1 = ex2_approx(m1 - M);
+            const size_t o = (size_t)row * kMaxSplits + t.split;
+            p.pm[o] = M * kLn2;  // back to natural units
+            p.pl[o] = run_l * w0 + xch[r_in_tile * 4 + 1] * w1;
+            p.ps[o] = run_s * w0 + xch[r_in_tile * 4 + 2] * w1;
+            p.pz[o] = run_z + xch[r_in_tile * 4 + 3];
+          }
+          epilogue_bar_all256();  // the exchange buffer may be written again
+        }
+        continue;
+      }
       if (KC::kWideSweep) {
         // This group's 128 columns of each accumulator, 32 at a time with the next 32 already
         // on their way from TMEM: exp, sums, bf16; each 32 columns leave through one of the

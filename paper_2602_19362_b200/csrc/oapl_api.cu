@@ -357,7 +357,8 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.n_live_ptr = &state->n_live;
   gp.row_begin = 0;
   gp.row_cap = c.n_pad;
-  pick_sweep(n_sm, p->d, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+  const int vtiles = (p->V + 2 * kBN - 1) / (2 * kBN);  // the sweep walks 512-column tiles
+  pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
   gp.d = p->d;
   gp.V = p->V;
   gp.pm = reinterpret_cast<float*>(ws + c.pm);
@@ -367,11 +368,11 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
   set_lockstep(&gp, ws, c, 0, p->d / kBK);
-  int rc = launch_gemm<MODE_LSE, 0, 0>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
+  int rc = launch_gemm<MODE_LSE, 0, 0, 2>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
-  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.ps, gp.R, gp.C, (p->V + kBN - 1) / kBN,
-                                             state, live_rows, lse, lp_c,
+  merge_lse_kernel<<<n_sm * 2, 256, 0, st>>>(gp.pm, gp.pl, gp.pz, gp.ps, gp.R, gp.C, vtiles, state, live_rows, lse,
+                                             lp_c,
                                              reinterpret_cast<float*>(ws + c.ent_c), token_logp);
   CKL();
   seq_sums_kernel<<<p->S, 256, 0, st>>>(lp_c, q_c, cstart, cend, seq_logp,
