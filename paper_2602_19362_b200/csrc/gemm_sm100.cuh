@@ -67,7 +67,8 @@ struct TileCfg {
 // Launch shape of one instantiation.
 template <int MODE, int NACC>
 struct KernelCfg {
-  static constexpr bool kWideSweep = (MODE == 5 /*MODE_LSE_E*/ && NACC == 2);
+  // sweeps that store a bf16 value per element: staged exponentials (MODE_LSE_E) or logit gradients (MODE_GRAD)
+  static constexpr bool kWideSweep = ((MODE == 5 || MODE == 1) && NACC == 2);
   static constexpr bool kWideLse = (MODE == 0 /*MODE_LSE*/ && NACC == 2);  // online log-sum-exp, no output tile
   static constexpr bool kReduceOut = (MODE == 3 /*MODE_DW*/ && NACC == 2);  // fp32 tile added by TMA
   static constexpr int kEpiWarps = (kWideSweep || kWideLse) ? 8 : 4;
@@ -311,8 +312,6 @@ template <int MODE, int A_MN, int B_MN, int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((KernelCfg<MODE, NACC>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const __grid_constant__ CUtensorMap tmC, const GemmParams p) {
-  static_assert(NACC == 1 || MODE != MODE_GRAD,
-                "this sweep is written for the alternating accumulators of the 256 x 256 tile");
   using Cfg = TileCfg<NACC>;
   using KC = KernelCfg<MODE, NACC>;
   constexpr int kStages = Cfg::kStages, kStageBytes = Cfg::kStageBytes;
@@ -680,6 +679,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // exp / sums / packing of one 32-column chunk into 16 words of w
         auto do_chunk = [&](const uint32_t (&r)[32], int c, uint32_t* w16) {
           const int col0 = t.n0 + chunk_off(c);
+          if (MODE == MODE_GRAD) {
+            // g = c * (onehot - exp(z - lse)); columns past V and rows past the range are 0
+            if (valid && col0 < p.V) {
+              const int ti = tgt - col0;
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                float g0 = -cf * ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -ref2));
+                float g1 = -cf * ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -ref2));
+                if (i == ti) g0 += cf;
+                if (i + 1 == ti) g1 += cf;
+                if (col0 + i >= p.V) g0 = 0.f;
+                if (col0 + i + 1 >= p.V) g1 = 0.f;
+                w16[i >> 1] = pack_bf16x2(g0, g1);
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) w16[i] = 0u;
+            }
+            return;
+          }
           if (valid && col0 < p.V) {
             const int ti = tgt - col0;
             float acc = 0.f, accs = 0.f;
@@ -743,7 +762,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
         }
-        if (t.last) {
+        if (MODE == MODE_LSE_E && t.last) {
           // end of this row block's sweep: group 1 hands its sums to group 0 through its piece
           float* xch = reinterpret_cast<float*>(out_smem + 2 * kPiece);
           if (group == 1) {

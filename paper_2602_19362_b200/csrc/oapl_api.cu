@@ -643,11 +643,12 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   CKL();
   if (!accumulate_dW) CK(cudaMemsetAsync(dW, 0, 4 * (size_t)p->V * (size_t)p->d, st));
 
-  CUtensorMap tmH, tmW, tmGk, tmWmn, tmGmn, tmHmn, tmdW;
+  CUtensorMap tmH, tmW, tmGk, tmGst, tmWmn, tmGmn, tmHmn, tmdW;
   const uint64_t ldg = (uint64_t)c.ldg;
   bool ok = make_map(&tmH, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmW, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 128) &&
             make_map(&tmGk, G, (uint64_t)c.chunk_rows, ldg, ldg, 128) &&
+            make_map_store32(&tmGst, G, (uint64_t)c.chunk_rows, ldg, ldg) &&
             make_map(&tmWmn, p->W, (uint64_t)p->V, (uint64_t)p->d, (uint64_t)p->d, 64) &&
             make_map(&tmGmn, G, (uint64_t)c.chunk_rows, ldg, ldg, 64) &&
             make_map(&tmHmn, Hc, (uint64_t)c.n_pad, (uint64_t)p->d, (uint64_t)p->d, 64) &&
@@ -671,7 +672,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   gp.dW = dW;
   gp.accumulate = 1;  // dW is zeroed above unless the caller accumulates; every chunk adds
   gp.err = &state->status;
-  pick_sweep(n_sm, p->d, (p->V + kBN - 1) / kBN, &gp.R, &gp.C);
+  pick_sweep(n_sm, p->d, (p->V + 2 * kBN - 1) / (2 * kBN), &gp.R, &gp.C);  // 512-column sweep tiles
 
   // Row chunks of the compacted rows.  The live-row count lives on the device, so the
   // host enqueues every chunk the row count N could need; chunks past the live rows
@@ -681,7 +682,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
     gp.row_begin = r0;
     set_lockstep(&gp, w, c, slot++, p->d / kBK);
-    rc = launch_gemm<MODE_GRAD, 0, 0>(tmH, tmW, tmGk, gp, 2 * gp.R * gp.C, st);
+    rc = launch_gemm<MODE_GRAD, 0, 0, 2>(tmH, tmW, tmGst, gp, 2 * gp.R * gp.C, st);
     if (rc != OAPL_OK) return rc;
     set_lockstep(&gp, w, c, slot++, 0);
     rc = launch_gemm<MODE_DH, 0, 1, 2>(tmGk, tmWmn, tmGk, gp, n_sm & ~1, st);
