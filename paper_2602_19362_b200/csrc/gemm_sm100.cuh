@@ -8,19 +8,19 @@
 //               sequences, per-row sum of e and target logit (no recompute in the backward)
 //   MODE_DEBUG  plain C = A.B for bring-up of the four operand-major combinations
 //
-// The kernel runs as pairs of CTAs (clusters of two, one pair per two SMs) that share
-// one 256 x 256 x 64 tile per step through tcgen05.mma.cta_group::2: each CTA loads its
-// own 128 rows of A and 128 of B's 256 columns (so every operand byte is fetched from L2
-// by one SM only, without multicast), the leader CTA's UMMA thread issues for both, and
-// each CTA's TMEM receives its 128 rows of the accumulator.
-// CTA = 6 warps: warp 0 issues TMA loads, warp 1 owns TMEM (and, in the leader, issues the
-// UMMAs), warps 2..5 are the epilogue (one TMEM lane quadrant each).
+// The kernel runs as pairs of CTAs (clusters of two, one pair per two SMs) that share one
+// tile per step through tcgen05.mma.cta_group::2: each CTA loads its own 128 rows of A and
+// 128 of every 256 columns of B (so every operand byte is fetched from L2 by one SM only,
+// without multicast), the leader CTA's UMMA thread issues for both, and each CTA's TMEM
+// receives its 128 rows of the accumulators.
+// Warp 0 issues TMA loads, warp 1 owns TMEM (and, in the leader, issues the UMMAs), the
+// remaining warps are the epilogue: four (one TMEM lane quadrant each) or, in the vocabulary
+// sweeps, eight (two per quadrant, each taking half of an accumulator's columns).
 //
 // Two tile shapes (template parameter NACC):
 //   NACC = 1  256 x 256 pair tile, six shared-memory stages of 32 KB per CTA, the two
 //             256-column fp32 accumulators in TMEM alternate so that the epilogue of tile j
-//             overlaps the main loop of tile j+1 (the vocabulary sweeps: short K = d, heavy
-//             epilogue).  bf16 tiles leave through shared memory and TMA stores.
+//             overlaps the main loop of tile j+1.  Only the bring-up GEMM uses it now.
 //   NACC = 2  256 x 512 pair tile: both accumulators belong to one tile and every A slab
 //             feeds two UMMAs, so a third less operand traffic from L2 per flop and half as
 //             many re-reads of the streamed operand from HBM; four stages of 48 KB.  The
@@ -28,10 +28,9 @@
 //             half-accumulator order hides: the epilogue drains accumulator 0 first and
 //             releases it, and the UMMA thread starts the next tile with accumulator 0's
 //             share of the first four K-steps while accumulator 1 is still being drained.
-//             dH (K = V) and dW (K = rows of the range) use it with the four epilogue warps;
-//             the single-call logits sweep (short K = d, exp and bf16 stores per element)
-//             uses it with eight epilogue warps, two per TMEM lane quadrant, each taking
-//             half of an accumulator's columns.
+//             dH (K = V) and dW (K = rows of the range) have long K loops and four epilogue
+//             warps; dW leaves through TMA reduce-add.  The vocabulary sweeps (short K = d,
+//             an exponential per element, bf16 stores in two of the three) have eight.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -58,7 +57,7 @@ template <int NACC>
 struct TileCfg {
   static constexpr int kStages = NACC == 2 ? 4 : 6;
   static constexpr int kStageBytes = kABytes + NACC * kBBytes;
-  static constexpr int kOutTotal = NACC == 2 ? 0 : 2 * kOutBytes;
+  static constexpr int kOutTotal = 0;
   static constexpr int kTileN = NACC * kBN;  // columns of one pair tile
   static constexpr size_t kSmemBytes =
       size_t(kStages) * kStageBytes + kOutTotal + 1024 /*align*/ + 256 /*barriers*/;
@@ -648,9 +647,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           epilogue_bar_all256();  // the exchange buffer may be written again
         }
-        continue;
-      }
-      if (KC::kWideSweep) {
+      } else if (KC::kWideSweep) {
         // This group's 128 columns of each accumulator, 32 at a time with the next 32 already
         // on their way from TMEM: exp, sums, bf16; each 32 columns leave through one of the
         // group's two swizzled pieces in shared memory and a TMA store (tmC has 128 x 32
@@ -781,9 +778,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           epilogue_bar_all256();  // group 1 may stage into its piece again
         }
-        continue;
-      }
-      if (KC::kReduceOut) {
+      } else if (KC::kReduceOut) {
         // dW += tile: 32 fp32 columns at a time through one of two swizzled 128 x 32 pieces in
         // shared memory and a TMA reduce-add (tmC maps dW), so the old values never travel to
         // the SM.  Every element of dW belongs to one tile of the launch and launches follow
@@ -825,72 +820,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
         }
-        continue;
-      }
-      if (MODE == MODE_GRAD || MODE == MODE_LSE_E) {
-        // bf16 output tile, 64 columns at a time: registers -> swizzled smem piece -> TMA store
-#pragma unroll 1
-        for (int g = 0; g < kBN / 64; ++g) {
-          uint32_t w[32];
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            uint32_t r[32];
-            tmem_ld32(taddr + g * 64 + h * 32, r);
-            tmem_ld_wait();
-            const int col0 = t.n0 + g * 64 + h * 32;
-            if (valid && col0 < p.V) {
-              const int ti = tgt - col0;
-              if (MODE == MODE_LSE_E) {
-                // columns past V hold z = 0 (zero-filled W rows): finite, and their e is cleared
-                float acc = 0.f, accs = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                  const float z0 = __uint_as_float(r[i]), z1 = __uint_as_float(r[i + 1]);
-                  float e0 = ex2_approx(fmaf(z0, kLog2e, -ref2));
-                  float e1 = ex2_approx(fmaf(z1, kLog2e, -ref2));
-                  if (col0 + i >= p.V) e0 = 0.f;
-                  if (col0 + i + 1 >= p.V) e1 = 0.f;
-                  acc += e0 + e1;
-                  accs = fmaf(e0, z0, fmaf(e1, z1, accs));
-                  w[h * 16 + (i >> 1)] = pack_bf16x2(e0, e1);
-                }
-                run_l += acc;
-                run_s += accs;
-                if (ti >= 0 && ti < 32) {
-#pragma unroll
-                  for (int i = 0; i < 32; ++i)
-                    if (i == ti) run_z = __uint_as_float(r[i]);
-                }
-              } else {
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                  float g0 = -cf * ex2_approx(fmaf(__uint_as_float(r[i]), kLog2e, -ref2));
-                  float g1 = -cf * ex2_approx(fmaf(__uint_as_float(r[i + 1]), kLog2e, -ref2));
-                  if (i == ti) g0 += cf;
-                  if (i + 1 == ti) g1 += cf;
-                  if (col0 + i >= p.V) g0 = 0.f;
-                  if (col0 + i + 1 >= p.V) g1 = 0.f;
-                  w[h * 16 + (i >> 1)] = pack_bf16x2(g0, g1);
-                }
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) w[h * 16 + i] = 0u;
-            }
-          }
-          uint8_t* piece = out_smem + (g & 1) * kOutBytes;
-          // the store that last read this piece (two pieces ago) must have drained it
-          if (issuer) tma_store_wait_read<1>();
-          epilogue_bar_sync();
-          stage_row_sw128(piece, r_in_tile, w);
-          fence_proxy_async_smem();
-          epilogue_bar_sync();
-          if (issuer) {
-            tma_store_2d(&tmC, smem_u32(piece), t.n0 + g * 64, t.m0 - row_begin + (int)rank * kBM);
-            tma_store_commit();
-          }
-        }
       } else {
+        // dH and the bring-up GEMM: 32 columns at a time, stored straight from registers
 #pragma unroll 1
         for (int c = 0; c < t.nh * (kBN / 32); ++c) {
           uint32_t r[32];
@@ -903,40 +834,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(0), 0));
           }
-          if (MODE == MODE_LSE) {
-            if (col0 < p.V) {
-              float v[32];
-#pragma unroll
-              for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-              if (col0 + 32 > p.V) {
-                // a large finite negative: its exponential is 0 and 0 * v stays 0 (no NaN)
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (col0 + i >= p.V) v[i] = -3.0e38f;
-              }
-              float cmax = v[0];
-#pragma unroll
-              for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
-              const float m2 = fmaxf(run_m2, cmax * kLog2e);
-              float acc = 0.f, accs = 0.f;
-#pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float e = ex2_approx(fmaf(v[i], kLog2e, -m2));
-                acc += e;
-                accs = fmaf(e, v[i], accs);
-              }
-              const float resc = ex2_approx(run_m2 - m2);
-              run_l = run_l * resc + acc;
-              run_s = run_s * resc + accs;
-              run_m2 = m2;
-              const int ti = tgt - col0;
-              if (ti >= 0 && ti < 32) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (i == ti) run_z = v[i];
-              }
-            }
-          } else if (MODE == MODE_DH) {
+          if (MODE == MODE_DH) {
             const int crow = row_begin + row;
             if (crow < row_end && col0 < p.d) {
               const float sc = p.rowscale ? p.rowscale[crow] : 1.f;
@@ -949,20 +847,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               for (int q = 0; q < 4; ++q)
                 dst[q] = make_uint4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
             }
-          } else if (MODE == MODE_DW) {
-            if (row < p.V && col0 < p.d) {
-              float4* dst = reinterpret_cast<float4*>(p.dW + (size_t)row * p.d + col0);
-#pragma unroll
-              for (int q = 0; q < 8; ++q) {
-                float4 x = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                       __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
-                if (p.accumulate) {
-                  const float4 y = dst[q];
-                  x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
-                }
-                dst[q] = x;
-              }
-            }
           } else {
             if (row < p.M && col0 < p.N) {  // N is a multiple of 8
               float4* dst = reinterpret_cast<float4*>(p.Cdbg + (size_t)row * p.N + col0);
@@ -974,25 +858,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
           }
         }
-      }
-      // accumulator drained: hand the TMEM buffer back to the UMMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (NACC == 1) {
-          mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
-        } else {
-          if (t.nh == 1) mbar_arrive_cluster(mapa_shared(tempty_bar(0), 0));
-          mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
-        }
-      }
-      if (MODE == MODE_LSE || MODE == MODE_LSE_E) {
-        if (t.last && valid) {
-          const size_t o = (size_t)row * kMaxSplits + t.split;
-          if (MODE == MODE_LSE) p.pm[o] = run_m2 * kLn2;  // back to natural units
-          p.pl[o] = run_l;
-          p.pz[o] = run_z;
-          p.ps[o] = run_s;
+        // accumulator drained: hand the TMEM buffer back to the UMMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (NACC == 1) {
+            mbar_arrive_cluster(mapa_shared(tempty_bar(buf), 0));
+          } else {
+            if (t.nh == 1) mbar_arrive_cluster(mapa_shared(tempty_bar(0), 0));
+            mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
+          }
         }
       }
     }
