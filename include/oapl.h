@@ -47,6 +47,16 @@ typedef enum {
                                         non-finite values); use oapl_loss_fwd + oapl_loss_bwd for such inputs */
 } oapl_status;
 
+/*
+ * Environment variables read at call time (tuning and testing; defaults in parentheses):
+ *   OAPL_STAGE_ROWS    rows of staged exponentials per range in the single-call paths (32768)
+ *   OAPL_CHUNK_ROWS    rows per logit-gradient chunk of oapl_loss_bwd (18944)
+ *   OAPL_SPLITS        vocabulary splits per wave of the logits sweeps (chosen from the L2 budget)
+ *   OAPL_L2_BUDGET_MB  L2 budget for the hidden-state blocks of one wave of a sweep (72)
+ *   OAPL_SYNC_EVERY    K-steps between the lock-step meetings of the CTA pairs (32; 0 = never)
+ * They change workspace sizes and schedules, never results beyond summation order across splits.
+ */
+
 /* flags */
 #define OAPL_FLAG_NONE 0
 #define OAPL_FLAG_FUSED 1 /* oapl_workspace_bytes: size the workspace for oapl_loss_fwd_bwd */

@@ -384,6 +384,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       // follows through the shared pipeline barriers)
       bool meet = p.sync_ctr != nullptr && p.sync_every > 0 && rank == 0;
       const uint64_t pol_keep = l2_policy_evict_last();
+      const uint64_t pol_stream_in = l2_policy_evict_first();
       const unsigned int npairs = gridDim.x >> 1;
       unsigned int epochs = 0;
       for (int j = 0; ok && get_tile<MODE, NACC>(p, row_begin, row_end, j, t); ++j) {
@@ -422,6 +423,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
                 for (int b = 0; b < kHalfN / 64; ++b)
                   tma_load_2d(sb + b * 8192, &tmB, fb, bn + 64 * b, kbb);
+              } else if (KC::kWideSweep || KC::kWideLse) {
+                // W streams through once per wave: it should not push the H blocks out of L2
+                tma_load_2d_hint(sb, &tmB, fb, kbb, bn, pol_stream_in);
               } else {
                 tma_load_2d(sb, &tmB, fb, kbb, bn);
               }
