@@ -354,6 +354,21 @@ def row_dH(h, W, target, c):
     return c * (g @ W)
 
 
+def vocab_rows_dW(vs, W_vs, H, targets, mask, seq_id, coef, lse):
+    """Rows vs of dL/dW at once (same definition as vocab_row_dW, one matrix
+    product for the logits of those vocabulary rows).  The result is additive
+    over row blocks of H, so a caller may sum it over chunks of rows."""
+    H = np.asarray(H, dtype=np.float64)
+    vs = np.asarray(vs).astype(np.int64)
+    m = np.asarray(mask).astype(np.float64)
+    Z = H @ np.asarray(W_vs, dtype=np.float64).T                      # [rows, len(vs)]
+    P = np.where(m[:, None] > 0, np.exp(Z - np.asarray(lse, dtype=np.float64)[:, None]), 0.0)
+    onehot = (np.asarray(targets).astype(np.int64)[:, None] == vs[None, :]).astype(np.float64)
+    c = np.asarray(coef, dtype=np.float64)[np.asarray(seq_id).astype(np.int64)] * m
+    G = c[:, None] * (onehot - P)
+    return G.T @ H
+
+
 def vocab_row_dW(v, w_v, H, targets, mask, seq_id, coef, lse):
     """dL/dW[v, :] given every live row's log-sum-exp.
 

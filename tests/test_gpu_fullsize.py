@@ -58,6 +58,31 @@ def test_full_size_sampled_rows_and_invariants(name, fused, beta):
     for i in range(len(rows)):
         assert hp.fro_rel(got[i], dH_ref[i]) <= 2 * hp.TOL_FRO
 
+    # --- sampled vocabulary rows of dW (the most frequent targets, the first and last rows, random
+    #     ones): z[n, v] of one vocabulary row costs O(N d), and the log-sum-exp of every live row
+    #     follows from the (sample-checked) token log-probs as z[n, y_n] - lp_n
+    if name == "7b" and fused:
+        gv = torch.Generator().manual_seed(2)
+        counts = torch.bincount(dev["targets"][mask].long(), minlength=V)
+        vs = torch.cat([torch.topk(counts, 8).indices.cpu(), torch.tensor([0, 1, 255, 256, V - 1]),
+                        torch.randint(0, V, (35,), generator=gv)]).unique()
+        W_vs = orc.bf16_bits_to_f64(synth.bf16_bits(dev["W"][vs.cuda()]))
+        live_idx = hp.npy(torch.nonzero(mask).flatten())
+        want = np.zeros((len(vs), d))
+        for c0 in range(0, len(live_idx), 32768):
+            idx = live_idx[c0:c0 + 32768]
+            it = torch.from_numpy(idx).cuda()
+            Hc = orc.bf16_bits_to_f64(synth.bf16_bits(dev["H"][it]))
+            tg_c = hp.npy(dev["targets"][it])
+            Wt = orc.bf16_bits_to_f64(synth.bf16_bits(dev["W"][torch.from_numpy(tg_c).long().cuda()]))
+            lse_c = np.einsum("nk,nk->n", Hc, Wt) - tok[idx]
+            want += orc.vocab_rows_dW(hp.npy(vs), W_vs, Hc, tg_c, np.ones(len(idx), dtype=np.uint8),
+                                      hp.npy(dev["seq_id"][it]), coef, lse_c)
+        got_w = hp.npy(out["dW"][vs.cuda()]).astype(np.float64)
+        assert hp.fro_rel(got_w, want) <= hp.TOL_FRO
+        for i in range(len(vs)):
+            assert hp.fro_rel(got_w[i], want[i]) <= 2 * hp.TOL_FRO, int(vs[i])
+
     # --- properties that hold at any size
     dH, dW = out["dH"], out["dW"]
     out.pop("ws")                               # the largest configuration needs the room for the checks

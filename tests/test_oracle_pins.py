@@ -298,6 +298,13 @@ def test_sampled_forms_agree_with_full_forms():
         row = orc.vocab_row_dW(v, p["W"][v], p["H"], p["targets"], p["mask"], p["seq_id"],
                                out["coef"], out["lse"])
         assert np.allclose(row, dW[v], atol=1e-12)
+    vs = [0, 5, 18, 3]
+    full = orc.vocab_rows_dW(vs, p["W"][vs], p["H"], p["targets"], p["mask"], p["seq_id"], out["coef"], out["lse"])
+    assert np.allclose(full, dW[vs], atol=1e-12)
+    half = len(p["mask"]) // 2                                           # additive over row blocks
+    parts = sum(orc.vocab_rows_dW(vs, p["W"][vs], p["H"][sl], p["targets"][sl], p["mask"][sl], p["seq_id"][sl],
+                                  out["coef"], out["lse"][sl]) for sl in (slice(0, half), slice(half, None)))
+    assert np.allclose(parts, dW[vs], atol=1e-12)
 
 
 def test_entropy_definition():
