@@ -310,7 +310,9 @@ def run_cuda(args) -> None:
         hbm = measured_peaks()["hbm"]
         adamw = {"elements": n_el, "ms": ms_a, "launches_per_step": (B.oapl_launch_count() - l0) // 8,
                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
-                              "traffic": None, "bytes_per_element": 34,
+                              # DRAM bytes measured by ncu on a 233 M-element weight, 33.8 per element,
+                              # scaled by the element count (profiles/adamw_kernels.md)
+                              "traffic": 33.8 * n_el, "bytes_per_element": 34,
                               "peak_kind": f"hbm_gbs of {measured_peaks()['source']}"}}
         del Wopt, master, m_st, v_st
 
