@@ -110,7 +110,6 @@ struct GemmParams {
   const int* live_rows;
   __nv_bfloat16* dH;  // [N, d]
   float* dW;          // [V, d]
-  int accumulate;
   // MODE_DEBUG
   float* Cdbg;
   int M, N, K;

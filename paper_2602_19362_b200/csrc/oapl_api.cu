@@ -473,7 +473,6 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   gp.live_rows = live_rows;
   gp.dH = static_cast<__nv_bfloat16*>(dH);
   gp.dW = dW;
-  gp.accumulate = 1;
   gp.err = &state->status;
   pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
 
@@ -670,7 +669,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   gp.live_rows = reinterpret_cast<int*>(w + c.live_rows);
   gp.dH = static_cast<__nv_bfloat16*>(dH);
   gp.dW = dW;
-  gp.accumulate = 1;  // dW is zeroed above unless the caller accumulates; every chunk adds
+  // dW is zeroed above unless the caller accumulates; every chunk adds to it
   gp.err = &state->status;
   pick_sweep(n_sm, p->d, (p->V + 2 * kBN - 1) / (2 * kBN), &gp.R, &gp.C);  // 512-column sweep tiles
 

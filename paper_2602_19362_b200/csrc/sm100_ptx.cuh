@@ -101,7 +101,8 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const void* tmap,
       "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x), "r"(y), "l"(policy)
       : "memory");
 }
-// tma_store_2d with an L2 eviction priority
+// 2-D tile store from shared memory (bulk async group) with an L2 eviction priority; the part of
+// the box outside the tensor is clipped.  x and y must not be negative.
 __device__ __forceinline__ void tma_store_2d_hint(const void* tmap, uint32_t src, int x, int y, uint64_t policy) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;" ::"l"(
                    reinterpret_cast<uint64_t>(tmap)),
@@ -130,17 +131,9 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
                : "memory");
 }
 
-// 2-D tile store from shared memory (bulk async group); the part of the box outside
-// the tensor is clipped.  x and y must not be negative.
-__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
-                   reinterpret_cast<uint64_t>(tmap)),
-               "r"(src), "r"(x), "r"(y)
-               : "memory");
-}
 // 2-D tile reduction into global memory: every fp32 element of the tile in shared memory is
 // added to the element of the tensor it maps to (performed by the memory system, nothing is read
-// back into the SM); same clipping and coordinate rules as the store.
+// back into the SM); same clipping and coordinate rules as the store above.
 __device__ __forceinline__ void tma_reduce_add_2d(const void* tmap, uint32_t src, int x, int y) {
   asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
                    reinterpret_cast<uint64_t>(tmap)),
