@@ -497,3 +497,49 @@ def test_adamw_closed_forms():
     _, m2, _, norm2 = orc.adamw_step(th, g, z, z, 1, 1e-2, 0.9, 0.95, 1e-8, 0.0, 0.5, other_sq_norm=100.0)
     assert norm2 == pytest.approx(math.sqrt((g * g).sum() + 100.0))
     assert np.allclose(m2, 0.1 * g * 0.5 / (norm2 + 1e-6), rtol=1e-12)
+
+
+# ---------------------------------------------------------------- autograd as an independent route
+def test_gradients_match_torch_autograd():
+    # Eq. 3 and the GRPO display typed out with torch ops in fp64 and differentiated by autograd:
+    # a different library and a different route (reverse mode through log_softmax) to dH and dW
+    import torch
+    p = _grpo_problem(5, noise=0.3)
+    Ht = torch.tensor(p["H"], dtype=torch.float64, requires_grad=True)
+    Wt = torch.tensor(p["W"], dtype=torch.float64, requires_grad=True)
+    tg = torch.tensor(p["targets"], dtype=torch.int64)
+    m = torch.tensor(p["mask"], dtype=torch.float64)
+    sid = torch.tensor(p["seq_id"], dtype=torch.int64)
+    lp = torch.log_softmax(Ht @ Wt.T, dim=1).gather(1, tg[:, None]).squeeze(1)
+
+    # OAPL: sum_i (beta2 * sum_t m (lp - q) - (r_i - vhat_g(i)))^2 with vhat from Eq. 2
+    beta_v, beta_loss, lam = 0.7, 0.3, 0.25
+    q = torch.tensor(p["logp_inf"], dtype=torch.float64)
+    r = torch.tensor(p["reward"], dtype=torch.float64)
+    gid = torch.tensor(p["group_id"], dtype=torch.int64)
+    D = torch.zeros(p["S"], dtype=torch.float64).index_add(0, sid, m * (lp - q))
+    vhat = torch.stack([beta_v * torch.log(torch.mean(torch.exp(r[gid == g] / beta_v))) for g in range(p["P"])])
+    loss = lam * torch.sum((beta_loss * D - (r - vhat[gid])) ** 2)
+    gH, gW = torch.autograd.grad(loss, (Ht, Wt), retain_graph=True)
+    out = orc.loss_fwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], p["group_id"], p["reward"],
+                       p["logp_inf"], p["S"], p["P"], beta_v, beta_loss, lam)
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    assert out["loss"] == pytest.approx(float(loss.detach()), rel=1e-12)
+    assert np.allclose(dH, gH.numpy(), rtol=1e-9, atol=1e-12) and np.allclose(dW, gW.numpy(), rtol=1e-9, atol=1e-12)
+
+    # GRPO: -lam * sum_i 1/|y_i| sum_t w_t min(r_t A_i, clip(r_t) A_i), w_t detached data
+    adv = torch.tensor(orc.group_advantage(p["reward"], p["group_id"], p["P"], 1e-6))
+    old = torch.tensor(p["logp_old"], dtype=torch.float64)
+    ratio = torch.exp(lp - old)
+    w = torch.exp(old - q)
+    A = adv[sid]
+    T = torch.zeros(p["S"], dtype=torch.float64).index_add(0, sid, m)
+    term = w * torch.minimum(ratio * A, torch.clamp(ratio, 0.8, 1.2) * A) * m / T[sid]
+    gloss = -lam * term.sum()
+    gH, gW = torch.autograd.grad(gloss, (Ht, Wt))
+    go = orc.grpo_fwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], p["logp_old"], p["logp_inf"],
+                      adv.numpy(), p["S"], 0.2, lam)
+    dH, dW = orc.token_coef_bwd(p["H"], p["W"], p["targets"], p["mask"], go["coef"])
+    assert go["loss"] == pytest.approx(float(gloss.detach()), rel=1e-12)
+    assert go["clipped"].any()
+    assert np.allclose(dH, gH.numpy(), rtol=1e-9, atol=1e-12) and np.allclose(dW, gW.numpy(), rtol=1e-9, atol=1e-12)
