@@ -72,8 +72,8 @@ struct KernelCfg {
   static constexpr bool kReduceOut = (MODE == 3 /*MODE_DW*/ && NACC == 2);  // fp32 tile added by TMA
   static constexpr int kEpiWarps = (kWideSweep || kWideLse) ? 8 : 4;
   static constexpr int kThreads = 64 + 32 * kEpiWarps;
-  // bf16 output pieces staged for TMA stores: two alternating 128 x 64 pieces in the 256 x 256
-  // sweeps; two alternating 128 x 32 pieces for each group of four epilogue warps in the wide one
+  // bf16 output pieces staged for TMA stores: two alternating 32 x 32 pieces (2 KB each) for each
+  // of the eight epilogue warps of a sweep
   // the dW tiles: two alternating 128 x 32 fp32 pieces
   static constexpr int kOutTotal =
       kWideSweep ? 4 * (kOutBytes / 2)
@@ -300,11 +300,8 @@ __device__ __forceinline__ bool epilogue_all(bool ok) {
       : "memory");
   return r != 0;
 }
-// Named barriers of the eight-warp epilogue: 1 = all 256 threads, 2 + g = the 128 threads of group g.
+// Named barrier 1 over the 256 threads of the eight-warp epilogue.
 __device__ __forceinline__ void epilogue_bar_all256() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void epilogue_bar_group(int g) {
-  asm volatile("bar.sync %0, 128;" ::"r"(2 + g) : "memory");
-}
 
 template <int MODE, int A_MN, int B_MN, int NACC>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((KernelCfg<MODE, NACC>::kThreads), 1)
@@ -652,26 +649,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       } else if (KC::kWideSweep) {
         // This group's 128 columns of each accumulator, 32 at a time with the next 32 already
-        // on their way from TMEM: exp, sums, bf16; each 32 columns leave through one of the
-        // group's two swizzled pieces in shared memory and a TMA store (tmC has 128 x 32
-        // boxes).  An accumulator is handed back to the UMMA warp as soon as this warp's last
-        // load from it has landed.
-        constexpr int kPiece = kOutBytes / 2;
+        // on their way from TMEM: exp, sums, bf16.  Every warp sends its own 32 rows x 32 columns
+        // through one of its two swizzled 2 KB pieces in shared memory and a TMA store of its own
+        // (tmC has 32 x 32 boxes), so the stores need no barrier between warps.  An accumulator
+        // is handed back to the UMMA warp as soon as this warp's last load from it has landed.
+        constexpr int kWarpPiece = 32 * 64;  // 32 rows of 32 bf16
+        uint8_t* const my_pieces = out_smem + (warp - 2) * (2 * kWarpPiece);
         const uint64_t pol_stream = l2_policy_evict_first();
         const int nchunks = 4 * t.nh;
-        // Stage 32 columns and send them off.  One barrier per piece: before it the issuing
-        // thread has seen every earlier store finish reading shared memory, so whoever passes
-        // it may overwrite the other buffer (last read by the previous piece's store) next time.
         auto send_chunk = [&](int c, const uint32_t* w16) {
-          uint8_t* piece = out_smem + (group * 2 + (c & 1)) * kPiece;
-          stage_row_sw64(piece, r_in_tile, w16);
+          uint8_t* piece = my_pieces + (c & 1) * kWarpPiece;
+          // lane 0 issues this warp's stores: the one two pieces back has drained this buffer
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+          stage_row_sw64(piece, lane, w16);
           fence_proxy_async_smem();
-          if (issuer) tma_store_wait_read<0>();
-          epilogue_bar_group(group);
-          if (issuer) {
-            // the staged exponentials are not read again before the whole range is written
+          __syncwarp();
+          if (lane == 0) {
+            // the staged values are not read again before the whole range is written
             tma_store_2d_hint(&tmC, smem_u32(piece), t.n0 + chunk_off_of(c, group),
-                              t.m0 - row_begin + (int)rank * kBM, pol_stream);
+                              t.m0 - row_begin + (int)rank * kBM + quad * 32, pol_stream);
             tma_store_commit();
           }
         };
@@ -763,23 +760,24 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
         }
         if (MODE == MODE_LSE_E && t.last) {
-          // end of this row block's sweep: group 1 hands its sums to group 0 through its piece
-          float* xch = reinterpret_cast<float*>(out_smem + 2 * kPiece);
+          // end of this row block's sweep: every warp of group 1 hands its rows' sums to the warp
+          // of group 0 that holds the same rows (four warps on), through its own first piece
+          float* xch = reinterpret_cast<float*>(out_smem + ((warp - 2) | 4) * (2 * kWarpPiece)) + lane * 4;
           if (group == 1) {
-            if (issuer) tma_store_wait_read<0>();
-            epilogue_bar_group(1);
-            xch[r_in_tile * 4 + 0] = run_l;
-            xch[r_in_tile * 4 + 1] = run_z;
-            xch[r_in_tile * 4 + 2] = run_s;
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
+            xch[0] = run_l;
+            xch[1] = run_z;
+            xch[2] = run_s;
           }
           epilogue_bar_all256();
           if (group == 0 && valid) {
             const size_t o = (size_t)row * kMaxSplits + t.split;
-            p.pl[o] = run_l + xch[r_in_tile * 4 + 0];
-            p.pz[o] = run_z + xch[r_in_tile * 4 + 1];
-            p.ps[o] = run_s + xch[r_in_tile * 4 + 2];
+            p.pl[o] = run_l + xch[0];
+            p.pz[o] = run_z + xch[1];
+            p.ps[o] = run_s + xch[2];
           }
-          epilogue_bar_all256();  // group 1 may stage into its piece again
+          epilogue_bar_all256();  // group 1 may stage into its pieces again
         }
       } else if (KC::kReduceOut) {
         // dW += tile: 32 fp32 columns at a time through one of two swizzled 128 x 32 pieces in
@@ -874,7 +872,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
       }
     }
-    if (issuer && (MODE == MODE_GRAD || MODE == MODE_LSE_E || KC::kReduceOut)) tma_store_wait_all();
+    // whoever issued bulk stores or reductions waits for them before the CTA may exit
+    if ((KC::kWideSweep && lane == 0) || (KC::kReduceOut && issuer)) tma_store_wait_all();
   }
 
   // ---------------------------------------------------------------- teardown

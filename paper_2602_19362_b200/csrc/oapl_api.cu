@@ -142,14 +142,14 @@ static bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t c
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The same matrix seen through 128-row x 32-column boxes (64-byte rows, 64-byte swizzle): the
-// store map of the wide logits sweep.
+// The same matrix seen through 32-row x 32-column boxes (64-byte rows, 64-byte swizzle): the
+// store map of the sweeps that write a bf16 value per element (one box per epilogue warp).
 static bool make_map_store32(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {ld * 2};
-  const cuuint32_t box[2] = {32, 128};
+  const cuuint32_t box[2] = {32, 32};
   const cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
