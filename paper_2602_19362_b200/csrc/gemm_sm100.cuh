@@ -604,22 +604,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               if (i == ti) run_z = v[i];
           }
         };
-        uint32_t ra[32], rb[32];
-        tmem_ld32(taddr + chunk_off_of(0, group), ra);
+        // all of this warp's 128 columns of an accumulator go to registers first, so the
+        // accumulator is handed back to the UMMA warp before the exponentials are taken
+        uint32_t rr[4][32];
+        (void)nchunks;
 #pragma unroll 1
-        for (int c = 0; c < nchunks; c += 2) {
+        for (int h = 0; h < t.nh; ++h) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tmem_ld32(taddr + chunk_off_of(4 * h + q, group), rr[q]);
           tmem_ld_wait();
-          tmem_ld32(taddr + chunk_off_of(c + 1, group), rb);
-          lse_chunk(ra, c);
-          tmem_ld_wait();
-          if (c + 2 < nchunks) tmem_ld32(taddr + chunk_off_of(c + 2, group), ra);
-          if (((c + 1) & 3) == 3) {
-            // that was this warp's last load from accumulator (c + 1) / 4
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) >> 2), 0));
-          }
-          lse_chunk(rb, c + 1);
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(h), 0));
+#pragma unroll
+          for (int q = 0; q < 4; ++q) lse_chunk(rr[q], 4 * h + q);
         }
         if (t.nh == 1) {
           __syncwarp();
@@ -736,24 +734,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             for (int i = 0; i < 16; ++i) w16[i] = 0u;
           }
         };
-        uint32_t ra[32], rb[32], w[16];
-        tmem_ld32(taddr + chunk_off(0), ra);
+        // All of this warp's 128 columns of an accumulator go to registers first, so the
+        // accumulator is handed back to the UMMA warp before the exponentials are taken.
+        uint32_t rr[4][32], w[16];
+        (void)nchunks;
 #pragma unroll 1
-        for (int c = 0; c < nchunks; c += 2) {
-          tmem_ld_wait();                                // chunk c is in ra
-          tmem_ld32(taddr + chunk_off(c + 1), rb);
-          do_chunk(ra, c, w);
-          send_chunk(c, w);
-          tmem_ld_wait();                                // chunk c + 1 is in rb
-          if (c + 2 < nchunks) tmem_ld32(taddr + chunk_off(c + 2), ra);
-          if (((c + 1) & 3) == 3) {
-            // that was this warp's last load from accumulator (c + 1) / 4
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar((c + 1) >> 2), 0));
+        for (int h = 0; h < t.nh; ++h) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tmem_ld32(taddr + chunk_off(4 * h + q), rr[q]);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(h), 0));
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            do_chunk(rr[q], 4 * h + q, w);
+            send_chunk(4 * h + q, w);
           }
-          do_chunk(rb, c + 1, w);
-          send_chunk(c + 1, w);
         }
         if (t.nh == 1) {
           __syncwarp();
