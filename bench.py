@@ -26,7 +26,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "response tokens/sec for OAPL loss fwd+bwd"
-MEASURED_DRAM_BYTES_PER_STEP = 737.9e9
+MEASURED_DRAM_BYTES_PER_STEP = 820.6e9
 UNIT = "tokens/s"
 
 
