@@ -24,6 +24,7 @@ static std::atomic<uint64_t> g_launches{0};
 constexpr int kChunkRowsDefault = 74 * 256;
 constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref) in the single-call path
 constexpr int kSyncSlots = 4096;             // lock-step counters in the workspace, one per contraction launch
+constexpr int kMaxDevices = 64;              // per-device host-side caches
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -171,13 +172,11 @@ static bool make_map_f32(CUtensorMap* m, const void* base, uint64_t rows, uint64
 }
 
 static int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 0;
-  }
-  return n;
+  static int n[kMaxDevices] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 0;
+  return n[dev];
 }
 
 // Sweep schedule: a wave is R row blocks (256 rows, one CTA pair each) x C vocabulary
@@ -243,14 +242,16 @@ static void prof_end(int slot, cudaStream_t st) {
 template <int MODE, int A_MN, int B_MN, int NACC = 1>
 static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
                        const GemmParams& gp, int grid, cudaStream_t st) {
-  static bool attr_set = false;
+  static bool attr_set[kMaxDevices] = {false};  // the attribute belongs to the function on one device
   auto kern = gemm_kernel<MODE, A_MN, B_MN, NACC>;
   constexpr size_t smem = KernelCfg<MODE, NACC>::kSmemBytes;
   constexpr int threads = KernelCfg<MODE, NACC>::kThreads;
-  if (!attr_set) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return OAPL_ERR_CUDA;
+  if (!attr_set[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return OAPL_ERR_CUDA;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   const int slot = prof_begin(MODE, st);
   if (slot >= 0 && g_prof_clk_addr) {
@@ -912,7 +913,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 
 // The array's name is only a host-side handle; kernels need its device address, which is
 // looked up once per device (with that device current) and cached.
-constexpr int kMaxDevices = 64;
 static unsigned char* g_static_scratch_addr[kMaxDevices] = {nullptr};
 
 static int static_scratch_for_current_device(unsigned char** out) {
