@@ -296,7 +296,9 @@ int oapl_profile_read_clocks(float* sm_mhz_by_kind /*host*/, int kinds);
  * [N, K] row-major; b_mn == 1: B is stored [K, N] row-major.  wide == 0: 256 x 256 tiles
  * with alternating accumulators (the vocabulary sweeps' shape); wide == 1: 256 x 512 tiles
  * (the shape of the dH and dW contractions).  K % 64 == 0, M % 8 == 0, N % 8 == 0.
- * `err` is a device int the kernel sets on a timeout.
+ * `err` points to TWO device ints: err[0] is set by the kernel on a timeout; err[1] is the
+ * counter of the CTA pairs' lock-step meetings (cleared by the call; OAPL_SYNC_EVERY=0
+ * switches the meetings off as in the other calls).
  */
 int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn,
                     int b_mn, int wide, int* err, void* stream);

@@ -225,6 +225,8 @@ def oapl_launch_count() -> int:
 
 
 def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err, wide=False):
+    if err is None or err.numel() < 2 or err.dtype != torch.int32:
+        raise TypeError("err: int32 CUDA tensor of two elements (status word, lock-step counter)")
     rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), int(wide), _ptr(err),
                                _stream())
     if rc != OAPL_OK:

@@ -876,6 +876,15 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   gp.K = K;
   gp.err = err;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    // the CTA pairs meet every 32 K-steps as in the product contractions
+    static const int forced = env_int("OAPL_SYNC_EVERY", -1);
+    if (forced != 0) {
+      CK(cudaMemsetAsync(err + 1, 0, sizeof(int), st));
+      gp.sync_ctr = reinterpret_cast<unsigned int*>(err + 1);
+      gp.sync_every = forced > 0 ? forced : 32;
+    }
+  }
   const int tile_n = wide ? 2 * kBN : kBN;
   const int tiles = ((M + kTileM - 1) / kTileM) * ((N + tile_n - 1) / tile_n);
   const int grid = 2 * (tiles < n_sm / 2 ? tiles : n_sm / 2);

@@ -21,10 +21,10 @@ def test_debug_gemm(M, N, K, a_mn, b_mn, wide):
     A_dev = (A.t().contiguous() if a_mn else A).cuda()
     B_dev = (Bm.t().contiguous() if b_mn else Bm).cuda()
     C = torch.full((M, N), float("nan"), device="cuda")
-    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    err = torch.zeros(2, dtype=torch.int32, device="cuda")     # status word, lock-step counter
     B.oapl_debug_gemm(A_dev, B_dev, C, M, N, K, a_mn, b_mn, err, wide=wide)
     torch.cuda.synchronize()
-    assert int(err.item()) == 0
+    assert int(err[0].item()) == 0
     got = C.cpu().numpy().astype(np.float64)
     assert np.isfinite(got).all()
     assert np.abs(got - ref).max() <= 1e-3 * np.sqrt(K) + 1e-3 * np.abs(ref).max()
