@@ -51,6 +51,24 @@ def run_gpu(dev, beta_v=None, beta_loss=None, loss_scale=None, backward=True, ac
     return out
 
 
+def run_gpu_async(dev, fused=True):
+    """Enqueue oapl_loss_fwd_bwd on the current stream without reading anything back (no
+    synchronisation), so that calls on different streams can overlap on the GPU."""
+    assert fused
+    prob = B.make_problem(dev)
+    ws = B.alloc_workspace(prob, B.OAPL_FLAG_FUSED)
+    N, S, P, d, V = (dev[k] for k in ("N", "S", "P", "d", "V"))
+    out = dict(loss=torch.zeros(1, device="cuda"), seq_logp=torch.zeros(S, device="cuda"),
+               vhat=torch.zeros(P, device="cuda"), delta=torch.zeros(S, device="cuda"),
+               token_logp=torch.zeros(N, device="cuda"),
+               dH=torch.empty(N, d, dtype=torch.bfloat16, device="cuda"),
+               dW=torch.empty(V, d, dtype=torch.float32, device="cuda"))
+    B.oapl_loss_fwd_bwd(prob, out["loss"], out["seq_logp"], out["vhat"], out["delta"], out["token_logp"],
+                        out["dH"], out["dW"], False, ws)
+    out["ws"], out["prob"] = ws, prob
+    return out
+
+
 def run_oracle(cpu, beta_v=None, beta_loss=None, loss_scale=None, backward=True):
     Hd = orc.bf16_bits_to_f64(synth.bf16_bits(cpu["H"]))
     Wd = orc.bf16_bits_to_f64(synth.bf16_bits(cpu["W"]))

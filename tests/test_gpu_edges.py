@@ -147,3 +147,24 @@ def test_single_call_reports_a_target_far_below_the_largest_logit():
     assert out["status"] == 0
     assert abs(float(out["token_logp"][row]) - ref["token_logp"][row]) <= hp.TOL_TOKEN
     hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
+
+
+def test_two_streams_with_their_own_workspaces_give_the_single_stream_results():
+    # Calls that overlap on the GPU compete for the SMs, so the CTA pairs of one launch may not all
+    # be resident when they try to meet: the meetings must give up quietly and results must not change.
+    wl = synth.small_variant("7b", prompts=2, samples=4, live_rows=450)
+    devs = [hp.to_dev(synth.make_batch(wl, seed=s)) for s in (21, 22)]
+    want = [hp.run_gpu(d, fused=True) for d in devs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [None, None]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for i, (d, st) in enumerate(zip(devs, streams)):
+            with torch.cuda.stream(st):
+                outs[i] = hp.run_gpu_async(d)
+        torch.cuda.synchronize()
+    for o, w in zip(outs, want):
+        assert B.oapl_get_last_status(o["ws"]) == 0
+        for k in ("loss", "seq_logp", "token_logp", "dW"):
+            assert torch.equal(o[k], w[k]), k
+        assert torch.equal(o["dH"].view(torch.int16), w["dH"].view(torch.int16))
