@@ -3,12 +3,17 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 7b] [--impl reference]
 
-A step is one oapl_loss_fwd_bwd call (Eq. 3 forward and gradient; `--path two-calls` times
+A step is one oapl_loss_fwd_bwd_ex call (Eq. 3 forward and gradient; `--path two-calls` times
 oapl_loss_fwd + oapl_loss_bwd instead) over one synthetic batch shaped like the paper's
 7B-scale trainer step (d=3584, V=152064, 16 prompts x 8 rollouts, response lengths
 U[512,4096], padded layout).  The metric is response tokens per second; the roofline
 object credits 6*N*d*V flops per step against the measured dense-bf16 peak.  Rank 0
 prints one JSON line.
+
+With --gpus N > 1 and no torchrun environment the script starts N ranks itself (one per GPU,
+torch.distributed.run on 127.0.0.1); every rank holds its own prompts (weak scaling, W
+replicated) and the step includes the NCCL all-reduce of dW, started on a second stream as
+soon as dW is complete, under the last range's dH contraction.
 """
 from __future__ import annotations
 
@@ -26,8 +31,13 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "response tokens/sec for OAPL loss fwd+bwd"
-MEASURED_DRAM_BYTES_PER_STEP = 820.6e9
 UNIT = "tokens/s"
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per live token of the three contraction
+# kinds of the single call, from one ncu capture of one launch per kind on a reduced copy of the
+# 7B workload (--prompts 1 --samples 4, 9.9 k live tokens, same d and V); the traffic of a kind
+# grows in proportion to the rows it processes, so a step's figure is this times its live tokens.
+# None = not captured for the present kernels.
+DRAM_BYTES_PER_TOKEN_7B = None
 
 
 # ---------------------------------------------------------------------------- helpers
@@ -126,6 +136,43 @@ def run_reference(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------- launcher
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_ranks(args) -> int:
+    """Started as plain `python bench.py --gpus N` (no torchrun environment): run the same
+    command line as N ranks under torch.distributed.run on this node and return its exit code."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, cwd=ROOT)
+
+
+def run_dry(args) -> None:
+    """Launcher check without a GPU: the ranks meet over gloo, aggregate a made-up per-rank time and
+    token count exactly as the timed arm does, and rank 0 prints a line marked as a dry run."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {world} rank(s) came up")
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms = reduce_max(10.0 + rank, dist if world > 1 else None, torch.device("cpu"))
+    tok = reduce_sum(1000.0, dist if world > 1 else None, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"dry_run": "launcher check only: no kernel ran, not a measurement", "metric": METRIC,
+                          "value": 0.0, "unit": UNIT, "n_gpus": world, "steps": 0, "warmup": 0,
+                          "ms_per_step": ms, "tokens_all_ranks": tok, "gpu_launches": 0}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------------------- CUDA arm
 def run_cuda(args) -> None:
     import torch
@@ -135,6 +182,11 @@ def run_cuda(args) -> None:
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but {world} rank(s) came up")
+    if not torch.cuda.is_available() or torch.cuda.device_count() < world:
+        raise SystemExit(f"{world} rank(s) need {world} CUDA device(s); {torch.cuda.device_count()} visible "
+                         "(there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -182,17 +234,32 @@ def run_cuda(args) -> None:
         B.oapl_group_advantage(batch["reward"], batch["group_id"], P, 1e-6, adv)
         clip_frac = torch.zeros(1, device=dev)
 
+    # what the host knows about the batch it built: the response-token count and the longest
+    # response bound the number of range slots the single call enqueues
+    comm_stream = torch.cuda.Stream() if world > 1 else None
+    dW_ready = None
+    if world > 1 and fused and not grpo:
+        dW_ready = torch.cuda.Event()
+        dW_ready.record()                      # torch creates the CUDA event at its first record
+    opts = B.make_options(live_rows_bound=n_live, max_seq_rows_bound=int(batch["lengths"].max()),
+                          dW_ready_event=dW_ready)
+
     def step(prob=prob, loss=loss, seq_logp=seq_logp, dH=dH, dW=dW):
         local_step(prob, loss, seq_logp, dH, dW)
         if world > 1:
             # the one exchange of the data-parallel step: sum of dW (and of the loss) over the ranks
-            dp.allreduce_outputs(loss, dW)
+            if dW_ready is not None:
+                # dW is complete before the last range's dH contraction: NCCL runs under it
+                handle = dp.start_allreduce_dW(dW, dW_ready, comm_stream)
+                dp.finish_allreduce(handle, loss)
+            else:
+                dp.allreduce_outputs(loss, dW)
 
     def local_step(prob, loss, seq_logp, dH, dW):
         if grpo:
             B.oapl_grpo_loss_fwd_bwd(prob, logp_old, adv, 0.2, loss, seq_logp, None, clip_frac, dH, dW, False, ws)
         elif fused:
-            B.oapl_loss_fwd_bwd(prob, loss, seq_logp, vhat, delta, None, dH, dW, False, ws)
+            B.oapl_loss_fwd_bwd_ex(prob, loss, seq_logp, vhat, delta, None, dH, dW, False, ws, opts)
         else:
             B.oapl_loss_fwd(prob, loss, seq_logp, vhat, delta, None, ws)
             B.oapl_loss_bwd(prob, dH, dW, False, ws)
@@ -226,8 +293,14 @@ def run_cuda(args) -> None:
     launches = B.oapl_launch_count() - launches0
     total_ms = ev[0].elapsed_time(ev[args.steps])
     step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
-    prof = B.oapl_profile_read()
+    prof, prof_dropped = B.oapl_profile_read(with_dropped=True)
     prof_mhz = B.oapl_profile_read_clocks()
+    n_ranges = B.oapl_get_range_count(ws) if fused else None
+    # the per-kind times are divided by the step count below: every step must have been recorded
+    n_rec = sum(v[1] for v in prof.values())
+    if prof_dropped or n_rec % args.steps:
+        raise RuntimeError(f"contraction timing incomplete: {n_rec} launches recorded over {args.steps} steps, "
+                           f"{prof_dropped} dropped")
     B.oapl_profile_enable(False)
     clocks = sampler.stop() if rank == 0 else None
     st = B.oapl_get_last_status(ws)
@@ -263,9 +336,10 @@ def run_cuda(args) -> None:
         hbm = measured_peaks()["hbm"]
         adamw = {"elements": n_el, "ms": ms_a, "launches_per_step": (B.oapl_launch_count() - l0) // 8,
                  "roofline": {"bound": "hbm", "achieved": gbs, "peak": hbm, "unit": "GB/s", "frac": gbs / hbm,
-                              # DRAM bytes measured by ncu on a 233 M-element weight, 33.8 per element,
-                              # scaled by the element count (profiles/adamw_kernels.md)
-                              "traffic": 33.8 * n_el, "bytes_per_element": 34,
+                              # DRAM bytes per element (33.8) measured by ncu on a 233 M-element weight,
+                              # scaled by the element count
+                              "traffic": 33.8 * n_el, "traffic_kind": "scaled from a reduced capture",
+                              "bytes_per_element": 34,
                               "peak_kind": f"hbm_gbs of {measured_peaks()['source']}"}}
         del Wopt, master, m_st, v_st
 
@@ -353,11 +427,11 @@ def run_cuda(args) -> None:
                 "executed_flops_per_step": exec_factor * n_live * d * V,
                 "achieved": exec_tflops, "peak": peak, "unit": "TFLOP/s",
                 "frac": exec_tflops / peak if exec_tflops else None,
-                # DRAM bytes of the contraction launches of one step of this workload
-                # (dram__bytes_read.sum + dram__bytes_write.sum, one ncu pass over the 102 launches of a
-                # step; profiles/gemm_kernel_7b.md); only valid for the default workload and path
-                "traffic": MEASURED_DRAM_BYTES_PER_STEP if (fused and not grpo and args.workload == "7b"
-                                                            and not (args.prompts or args.samples)) else None,
+                # DRAM bytes of the contraction launches of one step: the per-token figure of a reduced
+                # capture times this step's live tokens; only for the workload and path it was taken on
+                "traffic": (DRAM_BYTES_PER_TOKEN_7B * n_live
+                            if (DRAM_BYTES_PER_TOKEN_7B and fused and not grpo and args.workload == "7b") else None),
+                "traffic_kind": "scaled from a reduced capture (1 prompt x 4 rollouts, same d and V) by live tokens",
                 "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
                 "credited_tflops": flops_step / (ms_step * 1e-3) / 1e12,
                 "credited_frac_of_sustained": flops_step / (ms_step * 1e-3) / 1e12 / peaks["sustained"],
@@ -373,11 +447,18 @@ def run_cuda(args) -> None:
                                    f"lengths {wl.length}, padded_to={wl.padded_to}, beta={batch['beta_v']}",
                        "rows_N": N, "live_tokens_per_gpu": n_live, "parallelism": f"dp{world} over prompts" + (", NCCL all-reduce of dW and loss in the step" if world > 1 else ""),
                        "l2": "inputs larger than L2 (H, W, g chunk each > 126 MB); no flush needed",
-                       "api": ("oapl_grpo_loss_fwd_bwd" if grpo else "oapl_loss_fwd_bwd") if fused
+                       "api": ("oapl_grpo_loss_fwd_bwd" if grpo else "oapl_loss_fwd_bwd_ex") if fused
                               else "oapl_loss_fwd + oapl_loss_bwd",
+                       "host_bounds": None if (grpo or not fused) else
+                       {"live_rows_bound": n_live, "max_seq_rows_bound": int(batch["lengths"].max())},
+                       "ranges": n_ranges,
+                       "exchange": None if world == 1 else
+                       ("all-reduce of dW on a second stream behind the dW-ready event, under the last range's dH"
+                        if dW_ready is not None else "all-reduce of dW and loss after the call"),
                        "objective": args.objective,
                        "step_ms": step_ms, "loss": loss_val},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "gpu_launches_per_step": int(launches) // args.steps,
             "roofline": roofline, "cpu_baseline": cpu_base, "adamw_step": adamw}
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -403,10 +484,19 @@ def main() -> None:
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-adamw", action="store_true", help="skip the separately timed optimizer step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="launcher check on CPU (gloo): start the ranks, aggregate, print; no kernel runs")
     args = ap.parse_args()
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
-        run_reference(args)
+        run_reference(args)        # the oracle on host cores: rank 0 alone, whatever N
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    if args.dry_run:
+        run_dry(args)
     else:
         run_cuda(args)
 

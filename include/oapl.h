@@ -42,13 +42,16 @@ typedef enum {
   OAPL_ERR_CUDA = -9,                /* a CUDA runtime/driver call failed */
   OAPL_ERR_BAD_STATE = -10,          /* oapl_loss_bwd without a matching oapl_loss_fwd in ws */
   OAPL_ERR_SEQUENCE_TOO_LONG = -11,  /* device: oapl_loss_fwd_bwd met a sequence longer than its staging capacity */
-  OAPL_ERR_OUT_OF_RANGE = -12        /* device: a row's staged exponentials overflowed or vanished (single-call
+  OAPL_ERR_OUT_OF_RANGE = -12,       /* device: a row's staged exponentials overflowed or vanished (single-call
                                         paths: some logit exceeds the target's by more than ~128, or H / W hold
                                         non-finite values); use oapl_loss_fwd + oapl_loss_bwd for such inputs */
+  OAPL_ERR_BOUND_EXCEEDED = -13      /* device: the batch needs more ranges than the bounds passed in
+                                        oapl_call_options allow (more live rows, or a longer sequence) */
 } oapl_status;
 
 /*
- * Environment variables read at call time (tuning and testing; defaults in parentheses):
+ * Environment variables, read by every call that uses them (tuning and testing; defaults in
+ * parentheses):
  *   OAPL_STAGE_ROWS    rows of staged exponentials per range in the single-call paths (32768)
  *   OAPL_CHUNK_ROWS    rows per logit-gradient chunk of oapl_loss_bwd (18944)
  *   OAPL_SPLITS        vocabulary splits per wave of the logits sweeps (chosen from the L2 budget)
@@ -156,6 +159,38 @@ int oapl_loss_fwd_bwd(const oapl_problem* problem /*host*/, float* loss, float* 
                       int accumulate_dW, void* ws, size_t ws_bytes, int flags, void* stream);
 
 /*
+ * oapl_loss_fwd_bwd with what the caller knows about the batch on the host, and with a hook
+ * for the data-parallel trainer step (the paper trains with a global batch spread over several
+ * GPUs, "Experimental Details"; groups are independent in Eq. 2 / Eq. 3, so ranks hold whole
+ * groups and exchange only the sum of dW).
+ *
+ * The number of live rows exists only on the device, so the call enqueues as many range slots
+ * as the row count N could need; slots past the last range return at once.  A caller that
+ * built the batch knows better:
+ *   live_rows_bound     upper bound on the rows with mask==1 (0 = unknown: N is used);
+ *   max_seq_rows_bound  upper bound on the live rows of any one sequence (0 = unknown).
+ * They only reduce the number of (empty) launches.  Bounds that turn out too small are detected
+ * on the device: the status word becomes OAPL_ERR_BOUND_EXCEEDED and the outputs are not
+ * meaningful.
+ *   dW_ready_event      a cudaEvent_t (as void*) or NULL.  It is recorded on `stream` right after
+ *                       the last launch that writes dW; at that point the last range's dH
+ *                       contraction has not started yet.  A second stream that waits for the event
+ *                       can start the all-reduce of dW over the ranks under that contraction.
+ *                       loss, seq_logp and dH are complete only when `stream` is.
+ * options == NULL behaves like oapl_loss_fwd_bwd.
+ */
+typedef struct {
+  int64_t live_rows_bound;
+  int32_t max_seq_rows_bound;
+  void* dW_ready_event;
+} oapl_call_options;
+
+int oapl_loss_fwd_bwd_ex(const oapl_problem* problem /*host*/, float* loss, float* seq_logp, float* vhat,
+                         float* delta /*may be NULL*/, float* token_logp /*may be NULL*/, void* dH, float* dW,
+                         int accumulate_dW, void* ws, size_t ws_bytes, int flags,
+                         const oapl_call_options* options /*host, may be NULL*/, void* stream);
+
+/*
  * The paper's baseline objective on the same LM-head pass: GRPO reweighted by token-level
  * importance ratios (the display in the Background section),
  *     J = 1/G sum_{y in group} 1/|y| sum_t  w_t * min( r_t A, clip(r_t, 1-eps, 1+eps) A ),
@@ -237,6 +272,10 @@ int oapl_get_last_status(void* ws, void* stream);
  * synchronises `stream`.  Negative oapl_status on error. */
 int64_t oapl_get_live_rows(void* ws, void* stream);
 
+/* Number of ranges of whole sequences the last single call (oapl_loss_fwd_bwd,
+ * oapl_loss_fwd_bwd_ex, oapl_grpo_loss_fwd_bwd) on `ws` planned; synchronises `stream`. */
+int oapl_get_range_count(void* ws, void* stream);
+
 /* Kernel launches enqueued by this library in this process so far. */
 uint64_t oapl_launch_count(void);
 
@@ -269,24 +308,42 @@ const char* oapl_status_string(int status);
 int oapl_token_logprobs_static(const oapl_problem* problem /*host*/, float* token_logp, float* seq_logp,
                                int32_t* device_status, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Testing and timing aids.  Nothing below is part of the method; a trainer does not need it.
+ * ------------------------------------------------------------------------------------------ */
+
 /*
- * Optional timing of the contraction launches (off by default).  While enabled,
- * every contraction launch is bracketed by a CUDA event pair on its stream (at most
- * 2048 launches between reads).  oapl_profile_read waits for those events and sums
- * the elapsed milliseconds and the launch counts per kind into host arrays of
- * `kinds` entries: 0 = logits + online log-sum-exp, 1 = logit-gradient chunk,
- * 2 = dH, 3 = dW, 4 = bring-up GEMM, 5 = logits + staged exponentials; then clears the record.  Not thread-safe.
+ * Host logic only: the number of range slots the single call enqueues for a batch of at most
+ * live_rows_bound live rows in S sequences of at most max_seq_rows_bound live rows each
+ * (0 = unknown) and a staging capacity of stage_rows rows -- an upper bound on the number of
+ * ranges the greedy packing of whole sequences can produce.
+ */
+int oapl_range_slots(int64_t live_rows_bound, int64_t max_seq_rows_bound, int32_t stage_rows, int32_t S);
+
+/*
+ * Optional timing of the contraction launches (off by default).  oapl_profile_enable(1)
+ * switches it on for the CURRENT device: from then on every contraction launch on that device
+ * is bracketed by a CUDA event pair on its stream (launches on other devices run untimed).
+ * oapl_profile_read waits for those events and sums the elapsed milliseconds and the launch
+ * counts per kind into host arrays of `kinds` entries: 0 = logits + online log-sum-exp,
+ * 1 = logit-gradient chunk, 2 = dH, 3 = dW, 4 = bring-up GEMM, 5 = logits + staged
+ * exponentials; then clears the record.  At most 65536 launches are recorded between two
+ * reads; *launches_dropped (host, may be NULL) receives how many were not.  Not thread-safe.
  */
 int oapl_profile_enable(int on);
-int oapl_profile_read(float* ms_by_kind /*host*/, int* launches_by_kind /*host*/, int kinds);
+int oapl_profile_read(float* ms_by_kind /*host*/, int* launches_by_kind /*host*/, int kinds,
+                      int* launches_dropped /*host*/);
 /*
  * While the timing is enabled, CTA 0 of every contraction launch also adds its SM cycle count
- * and its elapsed nanoseconds to two per-kind device counters.  This call synchronises the
- * device, writes cycles/nanoseconds as MHz per kind (0 where the kind did not run) -- the SM
- * clock that kind of launch ran at, which on a power-capped part differs from kind to kind --
- * and clears the counters.  kinds <= 8.
+ * and its elapsed nanoseconds to two per-kind device counters.  This call (with the device the
+ * timing was enabled on current) synchronises the device, writes cycles/nanoseconds as MHz per
+ * kind (0 where the kind did not run) -- the SM clock that kind of launch ran at, which on a
+ * power-capped part differs from kind to kind -- and clears the counters.  kinds <= 8.
  */
 int oapl_profile_read_clocks(float* sm_mhz_by_kind /*host*/, int kinds);
+/* The rule the launches apply (host logic only, no CUDA call): 1 when a launch on
+ * `current_device` is timed given that the timing was enabled on `enabled_device` (-1 = off). */
+int oapl_profile_applies(int enabled_device, int current_device);
 
 /*
  * Bring-up aid for the tensor-core main loop shared by every contraction above:
@@ -294,14 +351,21 @@ int oapl_profile_read_clocks(float* sm_mhz_by_kind /*host*/, int kinds);
  * TMA/tcgen05 pipeline.  a_mn == 0: A is [M, K] row-major (K contiguous);
  * a_mn == 1: A is stored [K, M] row-major (M contiguous).  b_mn == 0: B is stored
  * [N, K] row-major; b_mn == 1: B is stored [K, N] row-major.  wide == 0: 256 x 256 tiles
- * with alternating accumulators (the vocabulary sweeps' shape); wide == 1: 256 x 512 tiles
- * (the shape of the dH and dW contractions).  K % 64 == 0, M % 8 == 0, N % 8 == 0.
- * `err` points to TWO device ints: err[0] is set by the kernel on a timeout; err[1] is the
- * counter of the CTA pairs' lock-step meetings (cleared by the call; OAPL_SYNC_EVERY=0
- * switches the meetings off as in the other calls).
+ * with alternating accumulators; wide == 1: 256 x 512 tiles (the shape of every product
+ * contraction).  K % 64 == 0, M % 8 == 0, N % 8 == 0.
+ * `err` points to TWO device ints: err[0] (cleared by the caller) is set by the kernel to
+ * OAPL_ERR_DEVICE_TIMEOUT when a pipeline wait gave up; err[1] is the counter of the CTA pairs'
+ * lock-step meetings (cleared by the call; OAPL_SYNC_EVERY=0 switches the meetings off).
+ *
+ * Test of the give-up path: wait_cycles > 0 replaces the limit of every pipeline wait (SM
+ * cycles; 0 = the product limit of 4e9), and skip_step = k > 0 makes the load warps leave out the
+ * loads of pipeline step k - 1, so that the wait for them runs out: every role then leaves its
+ * loop, the kernel frees its tensor memory and returns, and err[0] holds the timeout status
+ * (C is not meaningful).  skip_step needs 0 < wait_cycles <= 1e8.  Nothing faults and the
+ * context stays usable.
  */
 int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn,
-                    int b_mn, int wide, int* err, void* stream);
+                    int b_mn, int wide, long long wait_cycles, int skip_step, int* err, void* stream);
 
 #ifdef __cplusplus
 }

@@ -16,14 +16,16 @@ LIB_PATH = os.path.join(_HERE, "liboapl.so")
 OAPL_OK = 0
 STATUS = {0: "OK", -1: "INVALID_ARG", -2: "MISALIGNED", -3: "WORKSPACE_TOO_SMALL",
           -4: "UNSUPPORTED_SHAPE", -5: "BAD_TARGET", -6: "BAD_SEQ_ORDER", -7: "NONFINITE_INPUT",
-          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE", -11: "SEQUENCE_TOO_LONG", -12: "OUT_OF_RANGE"}
+          -8: "DEVICE_TIMEOUT", -9: "CUDA", -10: "BAD_STATE", -11: "SEQUENCE_TOO_LONG", -12: "OUT_OF_RANGE",
+          -13: "BOUND_EXCEEDED"}
 OAPL_FLAG_FUSED = 1
 
 EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate", "oapl_loss_fwd",
            "oapl_loss_bwd", "oapl_get_last_status", "oapl_get_live_rows", "oapl_launch_count",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
            "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy", "oapl_group_advantage",
-           "oapl_grpo_loss_fwd_bwd", "oapl_adamw_workspace_bytes", "oapl_adamw_step"]
+           "oapl_grpo_loss_fwd_bwd", "oapl_adamw_workspace_bytes", "oapl_adamw_step", "oapl_loss_fwd_bwd_ex",
+           "oapl_get_range_count", "oapl_profile_applies", "oapl_range_slots"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -33,6 +35,11 @@ class OaplProblem(ctypes.Structure):
                 ("mask", ctypes.c_void_p), ("seq_id", ctypes.c_void_p), ("group_id", ctypes.c_void_p),
                 ("reward", ctypes.c_void_p), ("logp_inf", ctypes.c_void_p),
                 ("beta_v", ctypes.c_float), ("beta_loss", ctypes.c_float), ("loss_scale", ctypes.c_float)]
+
+
+class OaplCallOptions(ctypes.Structure):
+    _fields_ = [("live_rows_bound", ctypes.c_int64), ("max_seq_rows_bound", ctypes.c_int32),
+                ("dW_ready_event", ctypes.c_void_p)]
 
 
 class OaplError(RuntimeError):
@@ -73,7 +80,16 @@ def lib() -> ctypes.CDLL:
         L.oapl_status_string.restype = ctypes.c_char_p
         L.oapl_status_string.argtypes = [i32]
         L.oapl_debug_gemm.restype = i32
-        L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp]
+        L.oapl_debug_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, ctypes.c_longlong, i32, vp, vp]
+        L.oapl_loss_fwd_bwd_ex.restype = i32
+        L.oapl_loss_fwd_bwd_ex.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32,
+                                           ctypes.POINTER(OaplCallOptions), vp]
+        L.oapl_get_range_count.restype = i32
+        L.oapl_get_range_count.argtypes = [vp, vp]
+        L.oapl_range_slots.restype = i32
+        L.oapl_range_slots.argtypes = [i64, i64, ctypes.c_int32, ctypes.c_int32]
+        L.oapl_profile_applies.restype = i32
+        L.oapl_profile_applies.argtypes = [i32, i32]
         L.oapl_loss_fwd_bwd.restype = i32
         L.oapl_loss_fwd_bwd.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, sz, i32, vp]
         L.oapl_token_logprobs_static.restype = i32
@@ -91,7 +107,7 @@ def lib() -> ctypes.CDLL:
         L.oapl_profile_enable.restype = i32
         L.oapl_profile_enable.argtypes = [i32]
         L.oapl_profile_read.restype = i32
-        L.oapl_profile_read.argtypes = [vp, vp, i32]
+        L.oapl_profile_read.argtypes = [vp, vp, i32, vp]
         L.oapl_profile_read_clocks.restype = i32
         L.oapl_profile_read_clocks.argtypes = [vp, i32]
         _lib = L
@@ -224,11 +240,11 @@ def oapl_launch_count() -> int:
     return int(lib().oapl_launch_count())
 
 
-def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err, wide=False):
+def oapl_debug_gemm(A, B, C, M, N, K, a_mn, b_mn, err, wide=False, wait_cycles=0, skip_step=0):
     if err is None or err.numel() < 2 or err.dtype != torch.int32:
         raise TypeError("err: int32 CUDA tensor of two elements (status word, lock-step counter)")
-    rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), int(wide), _ptr(err),
-                               _stream())
+    rc = lib().oapl_debug_gemm(_ptr(A), _ptr(B), _ptr(C), M, N, K, int(a_mn), int(b_mn), int(wide),
+                               int(wait_cycles), int(skip_step), _ptr(err), _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_debug_gemm")
 
@@ -242,14 +258,17 @@ def oapl_profile_enable(on: bool):
         raise OaplError(rc, "oapl_profile_enable")
 
 
-def oapl_profile_read() -> dict:
-    """{kind: (milliseconds, launches)} since the last read."""
+def oapl_profile_read(with_dropped: bool = False):
+    """{kind: (milliseconds, launches)} since the last read; with_dropped=True also returns the
+    number of launches that were not recorded."""
     ms = (ctypes.c_float * len(KINDS))()
     cnt = (ctypes.c_int * len(KINDS))()
-    rc = lib().oapl_profile_read(ms, cnt, len(KINDS))
+    dropped = ctypes.c_int(0)
+    rc = lib().oapl_profile_read(ms, cnt, len(KINDS), ctypes.byref(dropped))
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_profile_read")
-    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KINDS)}
+    out = {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KINDS)}
+    return (out, int(dropped.value)) if with_dropped else out
 
 
 def oapl_profile_read_clocks() -> dict:
@@ -268,6 +287,36 @@ def oapl_token_logprobs_static(problem, token_logp, seq_logp, device_status=None
                                           _ptr(device_status), _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_token_logprobs_static")
+
+
+def make_options(live_rows_bound: int = 0, max_seq_rows_bound: int = 0, dW_ready_event=None) -> OaplCallOptions:
+    """Fill oapl_call_options.  dW_ready_event is a torch.cuda.Event that has been recorded at
+    least once (torch creates the underlying CUDA event at the first record) or None."""
+    o = OaplCallOptions()
+    o.live_rows_bound = int(live_rows_bound)
+    o.max_seq_rows_bound = int(max_seq_rows_bound)
+    if dW_ready_event is None:
+        o.dW_ready_event = None
+    else:
+        handle = int(dW_ready_event.cuda_event)
+        if handle == 0:
+            raise ValueError("dW_ready_event: record the torch.cuda.Event once before passing it")
+        o.dW_ready_event = handle
+    return o
+
+
+def oapl_loss_fwd_bwd_ex(problem, loss, seq_logp, vhat, delta, token_logp, dH, dW, accumulate_dW, ws, options,
+                         flags=0):
+    rc = lib().oapl_loss_fwd_bwd_ex(ctypes.byref(problem), _ptr(loss), _ptr(seq_logp), _ptr(vhat), _ptr(delta),
+                                    _ptr(token_logp), _ptr(dH), _ptr(dW), int(accumulate_dW), _ptr(ws),
+                                    ws.numel(), flags, ctypes.byref(options) if options is not None else None,
+                                    _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_loss_fwd_bwd_ex")
+
+
+def oapl_get_range_count(ws) -> int:
+    return int(lib().oapl_get_range_count(_ptr(ws), _stream()))
 
 
 def oapl_loss_fwd_bwd(problem, loss, seq_logp, vhat, delta, token_logp, dH, dW, accumulate_dW, ws, flags=0):

@@ -121,6 +121,12 @@ struct GemmParams {
   // time those slabs live in L2.  The counter must be zero at launch.
   unsigned int* sync_ctr;
   int sync_every;
+  // Limit of every pipeline wait in SM cycles (0 = kWaitCycles, about 3 s).
+  long long wait_cycles;
+  // MODE_DEBUG only, for the test of the give-up path: the producers of every pair leave out
+  // the loads of pipeline step number test_skip_step - 1 (0 = none), so the consumers' wait
+  // for that step runs out.
+  int test_skip_step;
 };
 
 // Largest number of K-steps any CTA pair of this launch executes (all pairs compute the same
@@ -347,7 +353,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       row_end = p.row_begin + p.row_cap;
     }
     if (row_end > n_live) row_end = n_live;
+    // an empty row range (a range slot past the last planned range, a chunk past the live rows):
+    // every thread of both CTAs sees the same bounds and leaves before any barrier, TMEM or
+    // cluster set-up
+    if (row_end <= row_begin) return;
   }
+  const long long wlim = p.wait_cycles > 0 ? p.wait_cycles : kWaitCycles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -389,8 +400,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ++epochs;
             meet = lockstep_meet(p.sync_ctr, epochs * npairs);
           }
+          if (MODE == MODE_DEBUG && p.test_skip_step && it + 1 == (uint32_t)p.test_skip_step) continue;
           const int s = it % kStages;
-          if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag)) {
+          if (!mbar_wait(empty_bar(s), ((it / kStages) & 1u) ^ 1u, abort_flag, wlim)) {
             ok = false;
             break;
           }
@@ -447,7 +459,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         uint32_t d_tmem;
         if (NACC == 1) {
           const int buf = j & 1;
-          if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait(tempty_bar(buf), ((j >> 1) & 1u) ^ 1u, abort_flag, wlim)) break;
           d_tmem = tmem_base + buf * kBN;
         } else {
           d_tmem = tmem_base;
@@ -458,12 +470,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           // accumulator 0's UMMAs of the first `pre` K-steps (their stages are already loaded),
           // then wait for accumulator 1 and catch up on the same stages.
           const int pre = t.nk < kStages ? t.nk : kStages;
-          if (!mbar_wait(tempty_bar(0), (j & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait(tempty_bar(0), (j & 1u) ^ 1u, abort_flag, wlim)) break;
           tc_fence_after();
           for (int kb = 0; ok && kb < pre; ++kb) {
             const uint32_t itk = it + kb;
             const int s = itk % kStages;
-            if (!mbar_wait(full_bar(s), (itk / kStages) & 1u, abort_flag)) {
+            if (!mbar_wait(full_bar(s), (itk / kStages) & 1u, abort_flag, wlim)) {
               ok = false;
               break;
             }
@@ -480,7 +492,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             if (t.nh == 1) umma_commit_pair(empty_bar(s));
           }
           if (!ok) break;
-          if (!mbar_wait(tempty_bar(1), (j & 1u) ^ 1u, abort_flag)) break;
+          if (!mbar_wait(tempty_bar(1), (j & 1u) ^ 1u, abort_flag, wlim)) break;
           tc_fence_after();
           if (t.nh == 2) {
             for (int kb = 0; kb < pre; ++kb) {
@@ -504,7 +516,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         }
         for (int kb = kb_start; kb < t.nk; ++kb, ++it) {
           const int s = it % kStages;
-          if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag)) {
+          if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag, wlim)) {
             ok = false;
             break;
           }
@@ -561,7 +573,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           ref2 = p.lse[row] * kLog2e;
         }
       }
-      const bool got = mbar_wait(tfull_bar(buf), (NACC == 1 ? (j >> 1) : j) & 1u, abort_flag);
+      const bool got = mbar_wait(tfull_bar(buf), (NACC == 1 ? (j >> 1) : j) & 1u, abort_flag, wlim);
       if (!epilogue_all<32 * KC::kEpiWarps>(got)) break;
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + buf * kBN;

@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <vector>
 
 #include "../../include/oapl.h"
 #include "adamw.cuh"
@@ -89,7 +90,13 @@ static bool carve(const oapl_problem* p, int flags, Carve* c) {
     if ((size_t)stage > n_pad) stage = (int)n_pad;
     c->stage_rows = stage;
     c->stage_alloc_rows = stage + 256;
-    c->max_ranges = (int)(2 * n_pad / (size_t)stage) + 2;
+    // greedy packing of whole sequences: two neighbouring ranges together always hold more than
+    // `stage` rows, and every range holds at least one sequence
+    {
+      const size_t by_rows = 2 * ((n_pad + (size_t)stage - 1) / (size_t)stage) - 1;
+      c->max_ranges = (int)(by_rows < (size_t)p->S ? by_rows : (size_t)p->S);
+      if (c->max_ranges < 1) c->max_ranges = 1;
+    }
     c->G = take(2 * (size_t)c->stage_alloc_rows * (size_t)c->ldg);
     c->zref = take(4 * n_pad);
     c->alpha = take(4 * n_pad);
@@ -203,7 +210,7 @@ static void pick_sweep(int n_sm, int d, int vtiles, int* R, int* C) {
 // counter number `slot` of the workspace, which the caller has zeroed; every `nk_tile`-aligned
 // 32 K-steps or so.  OAPL_SYNC_EVERY overrides the interval (0 switches the meetings off).
 static void set_lockstep(GemmParams* gp, uint8_t* ws, const Carve& c, int slot, int nk_tile) {
-  static const int forced = env_int("OAPL_SYNC_EVERY", -1);
+  const int forced = env_int("OAPL_SYNC_EVERY", -1);
   gp->sync_ctr = nullptr;
   gp->sync_every = 0;
   if (forced == 0 || slot < 0 || slot >= kSyncSlots) return;
@@ -213,30 +220,55 @@ static void set_lockstep(GemmParams* gp, uint8_t* ws, const Carve& c, int slot, 
   gp->sync_every = every;
 }
 
-// Optional per-contraction timing (off by default): an event pair around every
-// contraction launch, summed per kind by oapl_profile_read.
-constexpr int kProfSlots = 2048;
-static bool g_prof_on = false;
-static int g_prof_used = 0;
-static cudaEvent_t g_prof_ev[kProfSlots][2];
-static int g_prof_kind[kProfSlots];
-static bool g_prof_made = false;
+// Optional per-contraction timing (off by default): an event pair around every contraction
+// launch on the device the timing was enabled on, summed per kind by oapl_profile_read.
+// Launches on any other device run untimed.  Event pairs are created as they are needed, up
+// to kProfMaxPairs between two reads; launches beyond that are counted as dropped.
+constexpr int kProfMaxPairs = 1 << 16;
+constexpr int kProfKinds = 8;
+struct ProfPair {
+  cudaEvent_t ev[2];
+  int kind;
+};
+struct ProfState {
+  int device = -1;               // device the timing is enabled on (-1 = off)
+  std::vector<ProfPair> pairs;   // pairs created so far (events belong to `made_on`)
+  int made_on = -1;
+  int used = 0;                  // pairs in use since the last read
+  int dropped = 0;               // launches not recorded since the last read
+  unsigned long long* clk_addr = nullptr;  // device address of g_prof_clk on `device`
+};
+static ProfState g_prof;
 
 // {SM cycles, nanoseconds} of CTA 0 of every contraction launch, summed per kind while
 // the timing is enabled; their ratio is the SM clock the kind ran at.
-constexpr int kProfKinds = 8;
 static __device__ unsigned long long g_prof_clk[kProfKinds][2];
-static unsigned long long* g_prof_clk_addr = nullptr;
 
-static int prof_begin(int kind, cudaStream_t st) {
-  if (!g_prof_on || g_prof_used >= kProfSlots) return -1;
-  const int s = g_prof_used++;
-  g_prof_kind[s] = kind;
-  cudaEventRecord(g_prof_ev[s][0], st);
+// Pure host logic of "is this launch timed": only on the device the timing was enabled on.
+static inline bool prof_applies(int enabled_device, int current_device) {
+  return enabled_device >= 0 && enabled_device == current_device;
+}
+
+static int prof_begin(int kind, int dev, cudaStream_t st) {
+  if (!prof_applies(g_prof.device, dev)) return -1;
+  if (g_prof.used >= (int)g_prof.pairs.size()) {
+    if ((int)g_prof.pairs.size() >= kProfMaxPairs) {
+      ++g_prof.dropped;
+      return -1;
+    }
+    ProfPair pr;
+    if (cudaEventCreate(&pr.ev[0]) != cudaSuccess) { ++g_prof.dropped; return -1; }
+    if (cudaEventCreate(&pr.ev[1]) != cudaSuccess) { cudaEventDestroy(pr.ev[0]); ++g_prof.dropped; return -1; }
+    pr.kind = 0;
+    g_prof.pairs.push_back(pr);
+  }
+  const int s = g_prof.used++;
+  g_prof.pairs[s].kind = kind;
+  cudaEventRecord(g_prof.pairs[s].ev[0], st);
   return s;
 }
 static void prof_end(int slot, cudaStream_t st) {
-  if (slot >= 0) cudaEventRecord(g_prof_ev[slot][1], st);
+  if (slot >= 0) cudaEventRecord(g_prof.pairs[slot].ev[1], st);
 }
 
 template <int MODE, int A_MN, int B_MN, int NACC = 1>
@@ -253,10 +285,10 @@ static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtenso
       return OAPL_ERR_CUDA;
     attr_set[dev] = true;
   }
-  const int slot = prof_begin(MODE, st);
-  if (slot >= 0 && g_prof_clk_addr) {
+  const int slot = prof_begin(MODE, dev, st);
+  if (slot >= 0 && g_prof.clk_addr) {
     GemmParams timed = gp;
-    timed.clk = g_prof_clk_addr + 2 * MODE;
+    timed.clk = g_prof.clk_addr + 2 * MODE;
     kern<<<grid, threads, smem, st>>>(a, b, c, timed);
   } else {
     kern<<<grid, threads, smem, st>>>(a, b, c, gp);
@@ -394,11 +426,35 @@ struct Objective {
   float* clip_frac;       // GRPO, may be null
 };
 
+// Number of range slots the single call enqueues: the largest number of ranges the greedy packing
+// of whole sequences into `stage` rows can produce for at most `live` live rows in sequences of at
+// most `longest` live rows each (0 = unknown), never more than the capacity of the range table.
+//   - two neighbouring ranges together hold more than `stage` rows:  n <= 2 ceil(live/stage) - 1
+//   - every range but the last holds more than stage - longest rows: n <= live/(stage-longest+1) + 1
+static int range_slots(long long live, long long longest, int stage, int S, int table_capacity) {
+  if (live < 1) live = 1;
+  long long n = 2 * ((live + stage - 1) / stage) - 1;
+  if (longest > 0 && longest <= stage) {
+    const long long m = live / (stage - longest + 1) + 1;
+    if (m < n) n = m;
+  }
+  if (n > S) n = S;
+  if (n > table_capacity) n = table_capacity;
+  if (n < 1) n = 1;
+  return (int)n;
+}
+
 static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* loss, float* seq_logp,
                           float* token_logp, void* dH, float* dW, int accumulate_dW, uint8_t* w,
-                          const Carve& c, cudaStream_t st) {
+                          const Carve& c, const oapl_call_options* opt, cudaStream_t st) {
   const int n_sm = sm_count();
   if (n_sm <= 0) return OAPL_ERR_CUDA;
+  long long live_bound = p->N, longest_bound = 0;
+  if (opt) {
+    if (opt->live_rows_bound > 0 && opt->live_rows_bound < live_bound) live_bound = opt->live_rows_bound;
+    longest_bound = opt->max_seq_rows_bound;
+  }
+  const int slots = range_slots(live_bound, longest_bound, c.stage_rows, p->S, c.max_ranges);
   int rc = prologue(p, c, w, token_logp, true, st);
   if (rc != OAPL_OK) return rc;
   DevState* state = reinterpret_cast<DevState*>(w + c.state);
@@ -445,7 +501,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   ztgt_kernel<<<n_sm * 8, 256, 0, st>>>(Hc, reinterpret_cast<const __nv_bfloat16*>(p->W), tgt_c, state,
                                         p->d, p->V, zref);
   CKL();
-  plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, c.max_ranges, ranges, state);
+  plan_ranges_kernel<<<1, 32, 0, st>>>(cstart, cend, p->S, c.stage_rows, slots, ranges, state);
   CKL();
 
   CUtensorMap tmH, tmW, tmEk, tmEst, tmWmn, tmEmn, tmHsmn, tmdW;
@@ -477,9 +533,11 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   gp.err = &state->status;
   pick_sweep(n_sm, p->d, vtiles, &gp.R, &gp.C);
 
-  // The ranges live on the device; the host enqueues the largest number of ranges the
-  // packing can produce and launches past the last range find no work.
-  for (int k = 0; k < c.max_ranges; ++k) {
+  // The ranges live on the device; the host enqueues the largest number of ranges the packing
+  // can produce for the row bounds it was given.  The planner fills the LAST slots, so empty
+  // slots come first (their launches return at once) and the last slot always holds the last
+  // range: the event after its dW launch marks dW complete while its dH contraction still runs.
+  for (int k = 0; k < slots; ++k) {
     const RangeRec* rg = ranges + k;
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
@@ -506,6 +564,8 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
     set_lockstep(&gp, w, c, 3 * k + 1, 0);
     rc = launch_gemm<MODE_DW, 1, 1, 2>(tmEmn, tmHsmn, tmdW, gp, n_sm & ~1, st);
     if (rc != OAPL_OK) return rc;
+    if (k == slots - 1 && opt && opt->dW_ready_event)
+      CK(cudaEventRecord(static_cast<cudaEvent_t>(opt->dW_ready_event), st));
     gp.rowscale = rowscale;
     set_lockstep(&gp, w, c, 3 * k + 2, 0);
     rc = launch_gemm<MODE_DH, 0, 1, 2>(tmEk, tmWmn, tmEk, gp, n_sm & ~1, st);
@@ -548,6 +608,7 @@ const char* oapl_status_string(int status) {
     case OAPL_ERR_BAD_STATE: return "backward called without a matching forward";
     case OAPL_ERR_SEQUENCE_TOO_LONG: return "a sequence has more live rows than the staging capacity";
     case OAPL_ERR_OUT_OF_RANGE: return "staged exponentials out of range (logit far above the target's, or non-finite input)";
+    case OAPL_ERR_BOUND_EXCEEDED: return "the batch has more live rows (or a longer sequence) than the caller's bounds";
     default: return "unknown status";
   }
 }
@@ -556,8 +617,6 @@ uint64_t oapl_launch_count(void) { return g_launches.load(std::memory_order_rela
 
 int oapl_get_last_status(void* ws, void* stream) {
   if (!ws) return OAPL_ERR_INVALID_ARG;
-  Carve dummy;
-  (void)dummy;
   DevState h;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return OAPL_ERR_CUDA;
@@ -572,6 +631,15 @@ int64_t oapl_get_live_rows(void* ws, void* stream) {
   if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return OAPL_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return OAPL_ERR_CUDA;
   return h.n_live;
+}
+
+int oapl_get_range_count(void* ws, void* stream) {
+  if (!ws) return OAPL_ERR_INVALID_ARG;
+  DevState h;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&h, ws, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return OAPL_ERR_CUDA;
+  return h.n_ranges;
 }
 
 int oapl_value_estimate(const float* reward, const int32_t* group_id, int32_t S, int32_t P,
@@ -697,9 +765,17 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
 int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float* vhat, float* delta,
                       float* token_logp, void* dH, float* dW, int accumulate_dW, void* ws,
                       size_t ws_bytes, int flags, void* stream) {
+  return oapl_loss_fwd_bwd_ex(p, loss, seq_logp, vhat, delta, token_logp, dH, dW, accumulate_dW, ws, ws_bytes,
+                              flags, nullptr, stream);
+}
+
+int oapl_loss_fwd_bwd_ex(const oapl_problem* p, float* loss, float* seq_logp, float* vhat, float* delta,
+                         float* token_logp, void* dH, float* dW, int accumulate_dW, void* ws,
+                         size_t ws_bytes, int flags, const oapl_call_options* options, void* stream) {
   int rc = check_problem(p, true);
   if (rc != OAPL_OK) return rc;
   if (!loss || !seq_logp || !vhat || !dH || !dW || !ws) return OAPL_ERR_INVALID_ARG;
+  if (options && (options->live_rows_bound < 0 || options->max_seq_rows_bound < 0)) return OAPL_ERR_INVALID_ARG;
   if (((uintptr_t)dH | (uintptr_t)dW) & 15) return OAPL_ERR_MISALIGNED;
   if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
   Carve c;
@@ -711,7 +787,7 @@ int oapl_loss_fwd_bwd(const oapl_problem* p, float* loss, float* seq_logp, float
   ob.vhat = vhat;
   ob.delta = delta;
   return staged_fwd_bwd(p, ob, loss, seq_logp, token_logp, dH, dW, accumulate_dW, static_cast<uint8_t*>(ws), c,
-                        static_cast<cudaStream_t>(stream));
+                        options, static_cast<cudaStream_t>(stream));
 }
 
 int oapl_group_advantage(const float* reward, const int32_t* group_id, int32_t S, int32_t P, float eps,
@@ -745,7 +821,7 @@ int oapl_grpo_loss_fwd_bwd(const oapl_problem* p, const float* logp_old, const f
   ob.clip_eps = clip_eps;
   ob.clip_frac = clip_frac;
   return staged_fwd_bwd(p, ob, loss, seq_logp, token_logp, dH, dW, accumulate_dW, static_cast<uint8_t*>(ws), c,
-                        static_cast<cudaStream_t>(stream));
+                        nullptr, static_cast<cudaStream_t>(stream));
 }
 
 size_t oapl_adamw_workspace_bytes(void) { return sizeof(double) * kAdamMaxPartials; }
@@ -814,51 +890,81 @@ int oapl_entropy(const oapl_problem* p, float* token_entropy, float* seq_entropy
 }
 
 int oapl_profile_enable(int on) {
-  if (on && !g_prof_made) {
-    for (int i = 0; i < kProfSlots; ++i)
-      for (int j = 0; j < 2; ++j)
-        if (cudaEventCreate(&g_prof_ev[i][j]) != cudaSuccess) return OAPL_ERR_CUDA;
-    g_prof_made = true;
+  if (!on) {
+    g_prof.device = -1;
+    g_prof.used = 0;
+    g_prof.dropped = 0;
+    return OAPL_OK;
   }
-  if (on) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_prof_clk) != cudaSuccess) return OAPL_ERR_CUDA;
-    g_prof_clk_addr = static_cast<unsigned long long*>(ptr);
-    if (cudaMemset(ptr, 0, sizeof(unsigned long long) * kProfKinds * 2) != cudaSuccess) return OAPL_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return OAPL_ERR_CUDA;
+  if (g_prof.made_on != dev) {
+    // events belong to the device they were created on: start over on another device
+    if (g_prof.made_on >= 0) {
+      int cur = dev;
+      if (cudaSetDevice(g_prof.made_on) == cudaSuccess)
+        for (auto& pr : g_prof.pairs) { cudaEventDestroy(pr.ev[0]); cudaEventDestroy(pr.ev[1]); }
+      cudaSetDevice(cur);
+    }
+    g_prof.pairs.clear();
+    g_prof.made_on = dev;
   }
-  g_prof_on = on != 0;
-  g_prof_used = 0;
+  void* ptr = nullptr;
+  if (cudaGetSymbolAddress(&ptr, g_prof_clk) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaMemset(ptr, 0, sizeof(unsigned long long) * kProfKinds * 2) != cudaSuccess) return OAPL_ERR_CUDA;
+  g_prof.clk_addr = static_cast<unsigned long long*>(ptr);
+  g_prof.device = dev;
+  g_prof.used = 0;
+  g_prof.dropped = 0;
   return OAPL_OK;
 }
 
 int oapl_profile_read_clocks(float* sm_mhz_by_kind, int kinds) {
   if (!sm_mhz_by_kind || kinds <= 0 || kinds > kProfKinds) return OAPL_ERR_INVALID_ARG;
-  if (!g_prof_clk_addr) return OAPL_ERR_BAD_STATE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (!g_prof.clk_addr || !prof_applies(g_prof.device, dev)) return OAPL_ERR_BAD_STATE;
   unsigned long long h[kProfKinds][2];
   if (cudaDeviceSynchronize() != cudaSuccess) return OAPL_ERR_CUDA;
-  if (cudaMemcpy(h, g_prof_clk_addr, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaMemcpy(h, g_prof.clk_addr, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) return OAPL_ERR_CUDA;
   for (int k = 0; k < kinds; ++k)
     sm_mhz_by_kind[k] = h[k][1] ? (float)((double)h[k][0] / (double)h[k][1] * 1e3) : 0.f;
-  if (cudaMemset(g_prof_clk_addr, 0, sizeof(h)) != cudaSuccess) return OAPL_ERR_CUDA;
+  if (cudaMemset(g_prof.clk_addr, 0, sizeof(h)) != cudaSuccess) return OAPL_ERR_CUDA;
   return OAPL_OK;
 }
 
-int oapl_profile_read(float* ms_by_kind, int* launches_by_kind, int kinds) {
+int oapl_profile_read(float* ms_by_kind, int* launches_by_kind, int kinds, int* launches_dropped) {
   if (!ms_by_kind || !launches_by_kind || kinds <= 0) return OAPL_ERR_INVALID_ARG;
   for (int k = 0; k < kinds; ++k) { ms_by_kind[k] = 0.f; launches_by_kind[k] = 0; }
-  for (int s = 0; s < g_prof_used; ++s) {
+  if (launches_dropped) *launches_dropped = g_prof.dropped;
+  for (int s = 0; s < g_prof.used; ++s) {
+    const ProfPair& pr = g_prof.pairs[s];
     float ms = 0.f;
-    if (cudaEventSynchronize(g_prof_ev[s][1]) != cudaSuccess) return OAPL_ERR_CUDA;
-    if (cudaEventElapsedTime(&ms, g_prof_ev[s][0], g_prof_ev[s][1]) != cudaSuccess) return OAPL_ERR_CUDA;
-    if (g_prof_kind[s] < kinds) { ms_by_kind[g_prof_kind[s]] += ms; launches_by_kind[g_prof_kind[s]] += 1; }
+    if (cudaEventSynchronize(pr.ev[1]) != cudaSuccess) return OAPL_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms, pr.ev[0], pr.ev[1]) != cudaSuccess) return OAPL_ERR_CUDA;
+    if (pr.kind < kinds) { ms_by_kind[pr.kind] += ms; launches_by_kind[pr.kind] += 1; }
   }
-  g_prof_used = 0;
+  g_prof.used = 0;
+  g_prof.dropped = 0;
   return OAPL_OK;
+}
+
+int oapl_range_slots(int64_t live_rows_bound, int64_t max_seq_rows_bound, int32_t stage_rows, int32_t S) {
+  if (stage_rows < 1 || S < 1 || live_rows_bound < 0 || max_seq_rows_bound < 0) return OAPL_ERR_INVALID_ARG;
+  return range_slots(live_rows_bound, max_seq_rows_bound, stage_rows, S, 0x7fffffff);
+}
+
+int oapl_profile_applies(int enabled_device, int current_device) {
+  return prof_applies(enabled_device, current_device) ? 1 : 0;
 }
 
 int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K, int a_mn, int b_mn,
-                    int wide, int* err, void* stream) {
-  if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return OAPL_ERR_INVALID_ARG;
+                    int wide, long long wait_cycles, int skip_step, int* err, void* stream) {
+  if (!A || !B || !C || !err || M <= 0 || N <= 0 || K <= 0) return OAPL_ERR_INVALID_ARG;
+  if (wait_cycles < 0 || skip_step < 0) return OAPL_ERR_INVALID_ARG;
+  // leaving a pipeline step out is only allowed together with a short wait limit (at most 1e8
+  // cycles, well under a tenth of a second), so that the launch ends soon
+  if (skip_step > 0 && (wait_cycles == 0 || wait_cycles > 100000000LL)) return OAPL_ERR_INVALID_ARG;
   if (K % 64 || M % 8 || N % 8) return OAPL_ERR_UNSUPPORTED_SHAPE;
   const int n_sm = sm_count();
   if (n_sm <= 0) return OAPL_ERR_CUDA;
@@ -875,10 +981,12 @@ int oapl_debug_gemm(const void* A, const void* B, float* C, int M, int N, int K,
   gp.N = N;
   gp.K = K;
   gp.err = err;
+  gp.wait_cycles = wait_cycles;
+  gp.test_skip_step = skip_step;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   {
     // the CTA pairs meet every 32 K-steps as in the product contractions
-    static const int forced = env_int("OAPL_SYNC_EVERY", -1);
+    const int forced = env_int("OAPL_SYNC_EVERY", -1);
     if (forced != 0) {
       CK(cudaMemsetAsync(err + 1, 0, sizeof(int), st));
       gp.sync_ctr = reinterpret_cast<unsigned int*>(err + 1);

@@ -39,12 +39,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
-// Every wait in the pipelines is bounded: after kWaitCycles without progress the
+// Every wait in the pipelines is bounded: after `limit` SM cycles without progress the
 // waiter raises the CTA-wide abort flag and returns false; all roles then leave
 // their loops, the kernel frees its TMEM and returns with an error word set.
+// kWaitCycles (about 3 s) is the limit of every product launch.
 constexpr long long kWaitCycles = 4000000000LL;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   uint32_t spins = 0;
   long long t0 = 0;
@@ -54,7 +56,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       long long now = clock64();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitCycles) {
+      } else if (now - t0 > limit) {
         *abort_flag = 1;
         return false;
       }

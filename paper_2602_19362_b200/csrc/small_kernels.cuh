@@ -18,6 +18,7 @@ struct DevState {
   int status;    // first device-detected error (0 = none)
   int fwd_tag;   // set by the forward, checked by the backward
   int ent_tag;   // set once the forward has left per-row entropies in the workspace
+  int n_ranges;  // single call: ranges of whole sequences planned by the last call
 };
 constexpr int kEntTag = 0x0E27;
 
@@ -345,35 +346,52 @@ __global__ void ztgt_kernel(const __nv_bfloat16* __restrict__ Hc, const __nv_bfl
 }
 
 // Greedy packing of consecutive sequences into ranges of at most stage_rows live rows.
-// One thread; S is small.  Unused records are left empty.  A sequence longer than
-// stage_rows cannot be staged: the error word is raised and no range is produced.
+// One thread; S is small.  The n ranges found occupy the LAST n of the max_ranges records (in
+// order), the records before them are left empty: the host enqueues max_ranges range slots
+// without knowing n, and the last slot is then always the last range.  A sequence longer
+// than stage_rows cannot be staged (-11), and more ranges than records means the caller's
+// bounds on the live rows were too small (-13): the error word is raised and no range is
+// produced.
 __global__ void plan_ranges_kernel(const int* __restrict__ cstart, const int* __restrict__ cend, int S,
                                    int stage_rows, int max_ranges, RangeRec* __restrict__ ranges,
                                    DevState* st) {
   if (blockIdx.x != 0 || threadIdx.x != 0) return;
-  for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
-  int n = 0, rb = -1, re = 0, sb = 0;
-  bool bad = false;
-  for (int s = 0; s < S && !bad; ++s) {
-    const int b = cstart[s], e = cend[s];
-    if (e <= b) continue;
-    if (e - b > stage_rows) { bad = true; break; }
-    if (rb < 0) { rb = b; sb = s; }
-    if (e - rb > stage_rows) {  // close the open range before this sequence
-      if (n < max_ranges) ranges[n] = RangeRec{rb, re, sb, s};
-      ++n;
-      rb = b;
-      sb = s;
+  for (int pass = 0; pass < 2; ++pass) {
+    // pass 0 counts the ranges, pass 1 writes them behind the empty records
+    int n = 0, rb = -1, re = 0, sb = 0;
+    const int shift = pass == 0 ? 0 : max_ranges - st->n_ranges;
+    for (int s = 0; s < S; ++s) {
+      const int b = cstart[s], e = cend[s];
+      if (e <= b) continue;
+      if (e - b > stage_rows) {
+        for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
+        set_error(&st->status, -11);
+        st->n_ranges = 0;
+        return;
+      }
+      if (rb < 0) { rb = b; sb = s; }
+      if (e - rb > stage_rows) {  // close the open range before this sequence
+        if (pass) ranges[shift + n] = RangeRec{rb, re, sb, s};
+        ++n;
+        rb = b;
+        sb = s;
+      }
+      re = e;
     }
-    re = e;
-  }
-  if (!bad && rb >= 0) {
-    if (n < max_ranges) ranges[n] = RangeRec{rb, re, sb, S};
-    ++n;
-  }
-  if (bad || n > max_ranges) {
-    for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
-    set_error(&st->status, bad ? -11 : -9);
+    if (rb >= 0) {
+      if (pass) ranges[shift + n] = RangeRec{rb, re, sb, S};
+      ++n;
+    }
+    if (pass == 0) {
+      if (n > max_ranges) {
+        for (int k = 0; k < max_ranges; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
+        set_error(&st->status, -13);
+        st->n_ranges = 0;
+        return;
+      }
+      st->n_ranges = n;
+      for (int k = 0; k < max_ranges - n; ++k) ranges[k] = RangeRec{0, 0, 0, 0};
+    }
   }
 }
 

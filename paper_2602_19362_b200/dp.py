@@ -57,3 +57,36 @@ def allreduce_outputs(loss: torch.Tensor, dW: torch.Tensor, group=None) -> None:
         return
     dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group)
     dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=group)
+
+
+def start_allreduce_dW(dW: torch.Tensor, dW_ready=None, comm_stream=None, group=None):
+    """Begin the sum of dW over the ranks while the step is still computing dH.
+
+    dW is complete before the single call's last dH contraction starts; the call records
+    `dW_ready` (a torch.cuda.Event) at that point.  On CUDA tensors the all-reduce is enqueued
+    on `comm_stream` behind that event, so NCCL runs under the remaining compute; on CPU
+    tensors (gloo) it is started asynchronously at once.  Returns a handle for
+    finish_allreduce; None without a process group."""
+    if not dist.is_available() or not dist.is_initialized() or dist.get_world_size(group) == 1:
+        return None
+    if dW.is_cuda:
+        if dW_ready is None or comm_stream is None:
+            raise ValueError("CUDA tensors need the dW-ready event and a communication stream")
+        with torch.cuda.stream(comm_stream):
+            comm_stream.wait_event(dW_ready)
+            dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group)
+        return ("cuda", comm_stream)
+    return ("cpu", dist.all_reduce(dW, op=dist.ReduceOp.SUM, group=group, async_op=True))
+
+
+def finish_allreduce(handle, loss: torch.Tensor, group=None) -> None:
+    """Sum the scalar loss over the ranks (it is complete only when the step's last kernel is)
+    and make the caller's stream wait for the dW exchange started by start_allreduce_dW."""
+    if handle is None:
+        return
+    dist.all_reduce(loss, op=dist.ReduceOp.SUM, group=group)
+    kind, h = handle
+    if kind == "cuda":
+        torch.cuda.current_stream().wait_stream(h)
+    else:
+        h.wait()

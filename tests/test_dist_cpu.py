@@ -88,6 +88,51 @@ def test_sharding_by_prompt_plus_allreduce_reproduces_the_single_rank_step():
     assert np.allclose(np.concatenate([g[7] for g in got]), ref["vhat"], rtol=1e-12)
 
 
+def _overlap_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    from paper_2602_19362_b200 import dp, synth
+    from tests import helpers_cpu as hc
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    full = synth.make_batch(hc.DP_WORKLOAD, seed=5)
+    ref = hc.oracle_step(dp.shard_by_prompt(full, rank, world))
+    # the exchange of the overlapped step: dW leaves as soon as it is complete, the rank goes on
+    # (here: it only then forms its loss tensor, as the device finishes dH and the loss after dW),
+    # and the scalar follows at the end
+    dW_a = torch.from_numpy(ref["dW"].copy())
+    handle = dp.start_allreduce_dW(dW_a)
+    loss_a = torch.tensor([ref["loss"]], dtype=torch.float64)
+    dp.finish_allreduce(handle, loss_a)
+    # the plain exchange after the step
+    dW_b, loss_b = torch.from_numpy(ref["dW"].copy()), torch.tensor([ref["loss"]], dtype=torch.float64)
+    dp.allreduce_outputs(loss_b, dW_b)
+    q.put((rank, bool(torch.equal(dW_a, dW_b)), float(loss_a), float(loss_b)))
+    dist.destroy_process_group()
+
+
+def test_exchange_started_when_dW_is_ready_equals_the_exchange_after_the_step():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 33500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_overlap_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=300) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert all(same for _, same, _, _ in got)
+    assert got[0][2] == got[0][3] == got[1][2] == got[1][3]
+
+
+def test_exchange_helpers_are_no_ops_without_a_process_group():
+    from paper_2602_19362_b200 import dp
+    dW, loss = torch.ones(4, 4), torch.ones(1)
+    assert dp.start_allreduce_dW(dW) is None
+    dp.finish_allreduce(None, loss)
+    assert float(dW.sum()) == 16.0 and float(loss) == 1.0
+
+
 def test_prompt_blocks_cover_every_prompt_once():
     from paper_2602_19362_b200 import dp
     for P, world in ((16, 8), (7, 3), (4, 4), (3, 5)):

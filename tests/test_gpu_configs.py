@@ -25,14 +25,18 @@ def test_small_variant_full_parity(name, rows):
     hp.assert_parity(out, ref, mask)
     # the single-call path (no recompute) on the same inputs
     hp.assert_parity(hp.run_gpu(dev, beta_v=betas[0], beta_loss=betas[0], fused=True), ref, mask)
-    # remaining temperatures of the sweep: forward quantities only need the cached
-    # oracle log-probs (Eq. 2 and Eq. 3 are O(S))
+    # remaining temperatures of the sweep, forward and backward on both paths: the oracle's forward
+    # quantities only need its cached log-probs (Eq. 2 and Eq. 3 are O(S)), its gradient is
+    # evaluated again with the new coefficients
+    Hd = orc.bf16_bits_to_f64(synth.bf16_bits(cpu["H"]))
+    Wd = orc.bf16_bits_to_f64(synth.bf16_bits(cpu["W"]))
     for b in betas[1:]:
-        o = hp.run_gpu(dev, beta_v=b, beta_loss=b, backward=False)
         r = orc.loss_from_sums(ref["D"], hp.npy(cpu["reward"]), hp.npy(cpu["group_id"]), cpu["P"], b, b,
                                cpu["loss_scale"])
         r.update(token_logp=ref["token_logp"], seq_logp=ref["seq_logp"], T=ref["T"])
-        hp.assert_parity(o, r, mask, backward=False)
+        r["dH"], r["dW"] = orc.loss_bwd(Hd, Wd, hp.npy(cpu["targets"]), mask, hp.npy(cpu["seq_id"]), r["coef"])
+        hp.assert_parity(hp.run_gpu(dev, beta_v=b, beta_loss=b), r, mask)
+        hp.assert_parity(hp.run_gpu(dev, beta_v=b, beta_loss=b, fused=True), r, mask)
     # the paper's own temperatures (beta_1 = 1 in Eq. 2, beta_2 = 1e-3 in Eq. 3)
     o = hp.run_gpu(dev, beta_v=1.0, beta_loss=1e-3, backward=False)
     r = orc.loss_from_sums(ref["D"], hp.npy(cpu["reward"]), hp.npy(cpu["group_id"]), cpu["P"], 1.0, 1e-3,

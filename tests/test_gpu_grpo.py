@@ -179,3 +179,8 @@ def test_7b_full_size_sampled_rows():
     assert float(out["dH"][~mask].float().abs().max()) == 0.0
     col = out["dW"].double().sum(dim=0)                      # softmax rows sum to 1
     assert float(col.abs().max()) <= 1e-3 * float(out["dW"].double().abs().sum(dim=0).max())
+    # sampled vocabulary rows of dW from the oracle's per-token coefficients
+    vs = hp.sample_vocab_rows(dev, mask, 50, seed=4)
+    assert vs.numel() >= 64
+    want_w, = hp.oracle_vocab_rows_dW(dev, mask, tok, vs, [ref["coef"]], per_token=True)
+    hp.assert_rows_close(hp.npy(out["dW"][vs.cuda()]).astype(np.float64), want_w, "grpo dW")
