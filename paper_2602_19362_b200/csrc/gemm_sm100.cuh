@@ -121,6 +121,10 @@ struct GemmParams {
   // time those slabs live in L2.  The counter must be zero at launch.
   unsigned int* sync_ctr;
   int sync_every;
+  // Vocabulary sweeps with 256 x 512 tiles: the last acc_skew K-steps of a tile are issued for
+  // accumulator 0 first, which is then handed to the epilogue while accumulator 1's share of those
+  // K-steps still runs (0 = both accumulators complete together; at most the stage count).
+  int acc_skew;
   // Limit of every pipeline wait in SM cycles (0 = kWaitCycles, about 3 s).
   long long wait_cycles;
   // MODE_DEBUG only, for the test of the give-up path: the producers of every pair leave out
@@ -514,7 +518,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         } else {
           tc_fence_after();
         }
-        for (int kb = kb_start; kb < t.nk; ++kb, ++it) {
+        // the last `post` K-steps of a sweep tile: accumulator 0 first (see GemmParams::acc_skew)
+        int post = 0;
+        if (NACC == 2 && (KC::kWideSweep || KC::kWideLse) && t.nh == 2) {
+          post = p.acc_skew < kStages ? p.acc_skew : kStages;
+          if (post > t.nk - kb_start) post = t.nk - kb_start;
+          if (post < 0) post = 0;
+        }
+        const int kb_end = t.nk - post;
+        for (int kb = kb_start; kb < kb_end; ++kb, ++it) {
           const int s = it % kStages;
           if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag, wlim)) {
             ok = false;
@@ -538,8 +550,42 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           }
           umma_commit_pair(empty_bar(s));  // both CTAs' stage reusable once these UMMAs have read it
         }
-        // accumulator(s) complete in both CTAs
-        if (ok) umma_commit_pair(tfull_bar(NACC == 1 ? (j & 1) : 0));
+        if (!ok) break;
+        if (NACC == 2 && post > 0) {
+          for (int q = 0; ok && q < post; ++q) {
+            const uint32_t itk = it + q;
+            const int s = itk % kStages;
+            if (!mbar_wait(full_bar(s), (itk / kStages) & 1u, abort_flag, wlim)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes;
+#pragma unroll
+            for (int kk = 0; kk < kBK / 16; ++kk)
+              umma_bf16(d_tmem, smem_desc_sw128(sa + kk * 32, 16, 1024), smem_desc_sw128(sb + kk * 32, 16, 1024),
+                        idesc, 1u);
+          }
+          if (!ok) break;
+          umma_commit_pair(tfull_bar(0));  // accumulator 0 complete in both CTAs
+          for (int q = 0; q < post; ++q) {
+            const int s = (it + q) % kStages;
+            const uint32_t sa = base + s * kStageBytes, sb = sa + kABytes + kBBytes;
+#pragma unroll
+            for (int kk = 0; kk < kBK / 16; ++kk)
+              umma_bf16(d_tmem + kBN, smem_desc_sw128(sa + kk * 32, 16, 1024),
+                        smem_desc_sw128(sb + kk * 32, 16, 1024), idesc, 1u);
+            umma_commit_pair(empty_bar(s));
+          }
+          it += post;
+          umma_commit_pair(tfull_bar(1));  // accumulator 1 complete
+        } else if (NACC == 2 && (KC::kWideSweep || KC::kWideLse)) {
+          umma_commit_pair(tfull_bar(0));
+          umma_commit_pair(tfull_bar(1));
+        } else {
+          // accumulator(s) complete in both CTAs
+          umma_commit_pair(tfull_bar(NACC == 1 ? (j & 1) : 0));
+        }
       }
     }
   } else {
@@ -620,8 +666,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // accumulator is handed back to the UMMA warp before the exponentials are taken
         uint32_t rr[4][32];
         (void)nchunks;
+        bool dead = false;
 #pragma unroll 1
         for (int h = 0; h < t.nh; ++h) {
+          if (h == 1) {
+            // accumulator 1 may complete later than accumulator 0 (GemmParams::acc_skew)
+            const bool got1 = mbar_wait(tfull_bar(1), j & 1u, abort_flag, wlim);
+            if (!epilogue_all<32 * KC::kEpiWarps>(got1)) {
+              dead = true;
+              break;
+            }
+            tc_fence_after();
+          }
 #pragma unroll
           for (int q = 0; q < 4; ++q) tmem_ld32(taddr + chunk_off_of(4 * h + q, group), rr[q]);
           tmem_ld_wait();
@@ -631,6 +687,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 #pragma unroll
           for (int q = 0; q < 4; ++q) lse_chunk(rr[q], 4 * h + q);
         }
+        if (dead) break;
         if (t.nh == 1) {
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));
@@ -750,8 +807,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         // accumulator is handed back to the UMMA warp before the exponentials are taken.
         uint32_t rr[4][32], w[16];
         (void)nchunks;
+        bool dead = false;
 #pragma unroll 1
         for (int h = 0; h < t.nh; ++h) {
+          if (h == 1) {
+            // accumulator 1 may complete later than accumulator 0 (GemmParams::acc_skew)
+            const bool got1 = mbar_wait(tfull_bar(1), j & 1u, abort_flag, wlim);
+            if (!epilogue_all<32 * KC::kEpiWarps>(got1)) {
+              dead = true;
+              break;
+            }
+            tc_fence_after();
+          }
 #pragma unroll
           for (int q = 0; q < 4; ++q) tmem_ld32(taddr + chunk_off(4 * h + q), rr[q]);
           tmem_ld_wait();
@@ -764,6 +831,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             send_chunk(4 * h + q, w);
           }
         }
+        if (dead) break;
         if (t.nh == 1) {
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty_bar(1), 0));

@@ -190,12 +190,18 @@ static int sm_count() {
 // splits, R*C <= number of CTA pairs.  C is the smallest power of two that keeps the wave's
 // H row blocks within an L2 budget; a short row range is handled by the tail-wave
 // re-splitting of the schedule itself.
+// The budget: every H block is re-read by its C pairs for each vocabulary tile and has to stay
+// in L2 for a whole sweep.  DRAM counters show that blocks read by pairs in both halves of the
+// chip take room in both halves of the 126 MB L2: with 68 MB of blocks (R = 37 at d = 3584) half
+// of the re-reads went to DRAM (22 GB read per 32 k rows against 4 GB needed), with 33 MB
+// (R = 18) almost none (10 GB against 8).
+constexpr int kL2BudgetMB = 48;
 static void pick_sweep(int n_sm, int d, int vtiles, int* R, int* C) {
   const int pairs = n_sm / 2;
   int c = env_int("OAPL_SPLITS", 0);
   if (c <= 0) {
     c = 1;
-    const size_t budget = (size_t)env_int("OAPL_L2_BUDGET_MB", 72) << 20;
+    const size_t budget = (size_t)env_int("OAPL_L2_BUDGET_MB", kL2BudgetMB) << 20;
     while (c < kMaxSplits && (size_t)(pairs / c) * kSweepRows * d * 2 > budget) c *= 2;
   }
   if (c > kMaxSplits) c = kMaxSplits;
@@ -273,7 +279,9 @@ static void prof_end(int slot, cudaStream_t st) {
 
 template <int MODE, int A_MN, int B_MN, int NACC = 1>
 static int launch_gemm(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
-                       const GemmParams& gp, int grid, cudaStream_t st) {
+                       const GemmParams& gp_in, int grid, cudaStream_t st) {
+  GemmParams gp = gp_in;
+  gp.acc_skew = env_int("OAPL_ACC_SKEW", TileCfg<NACC>::kStages);
   static bool attr_set[kMaxDevices] = {false};  // the attribute belongs to the function on one device
   auto kern = gemm_kernel<MODE, A_MN, B_MN, NACC>;
   constexpr size_t smem = KernelCfg<MODE, NACC>::kSmemBytes;
