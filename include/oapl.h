@@ -52,7 +52,7 @@ typedef enum {
 /*
  * Environment variables, read by every call that uses them (tuning and testing; defaults in
  * parentheses):
- *   OAPL_STAGE_ROWS    rows of staged exponentials per range in the single-call paths (32768)
+ *   OAPL_STAGE_ROWS    rows of staged exponentials per range in the single-call paths (65536)
  *   OAPL_CHUNK_ROWS    rows per logit-gradient chunk of oapl_loss_bwd (18944)
  *   OAPL_SPLITS        vocabulary splits per wave of the logits sweeps (chosen from the L2 budget)
  *   OAPL_L2_BUDGET_MB  L2 budget for the hidden-state blocks of one wave of a sweep (48)
@@ -147,7 +147,7 @@ int oapl_loss_bwd(const oapl_problem* problem /*host*/, void* dH, float* dW, int
  * lowered by sum_v e) both gradient contractions read the staged e' directly:
  * dH = rowscale(e'.W), dW += e'^T.(scaled H).  Executed work is 6*N*d*V flops instead of 8.
  *
- * Workspace: oapl_workspace_bytes(problem, OAPL_FLAG_FUSED).  It holds e for 32768 rows
+ * Workspace: oapl_workspace_bytes(problem, OAPL_FLAG_FUSED).  It holds e for 65536 rows
  * (2 bytes * round_up(V,512) each; OAPL_STAGE_ROWS in the environment changes the count), so
  * it does not grow with N*V; a sequence with more live rows than that cannot be staged and
  * raises OAPL_ERR_SEQUENCE_TOO_LONG in the status word (outputs are then not meaningful;

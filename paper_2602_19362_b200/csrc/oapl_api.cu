@@ -23,7 +23,9 @@ static std::atomic<uint64_t> g_launches{0};
 // rows of one g chunk of the two-call backward: 74 row blocks of 256, so that on 74 CTA pairs the
 // chunk's dH tiles (74 x d/512) fill whole rounds and its sweep two whole waves of 37 row blocks
 constexpr int kChunkRowsDefault = 74 * 256;
-constexpr int kStageRowsDefault = 32768;     // rows of staged e = exp(z - zref) in the single-call path
+// rows of staged e = exp(z - zref) per range in the single-call path (20 GB at V = 152064): the longer
+// the ranges, the fewer partial rounds of dH tiles, passes over dW and tail waves of the sweep
+constexpr int kStageRowsDefault = 65536;
 constexpr int kSyncSlots = 4096;             // lock-step counters in the workspace, one per contraction launch
 constexpr int kMaxDevices = 64;              // per-device host-side caches
 

@@ -135,7 +135,8 @@ def test_range_slot_bound_covers_the_greedy_packing(L):
         assert n <= L.oapl_range_slots(live, max(lens), stage, S), (lens, stage)
         assert n <= L.oapl_range_slots(live, 0, stage, S), (lens, stage)
         assert n <= L.oapl_range_slots(live + 5000, 0, stage, S)
-    # the 7B-scale benchmark batch: 309040 response tokens, sequences up to 4096, 32768-row staging
+    # the 7B-scale benchmark batch: 309040 response tokens, sequences up to 4096
+    assert L.oapl_range_slots(309040, 4096, 65536, 128) == 6
     assert L.oapl_range_slots(309040, 4096, 32768, 128) == 11
     assert L.oapl_range_slots(524288, 0, 32768, 128) == 31
     assert L.oapl_range_slots(10, 0, 32768, 128) == 1
