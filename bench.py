@@ -34,11 +34,11 @@ METRIC = "response tokens/sec for OAPL loss fwd+bwd"
 UNIT = "tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per live token of the single call's
 # three contraction kinds: one ncu capture of one launch per kind on a reduced copy of the 7B
-# workload that fills one range of whole sequences (--prompts 1 --samples 13 --seed 1: 32,634 live
-# tokens, same d and V): logits 9.96 + 10.12 GB, dW 26.25 + 2.17 GB, dH 25.00 + 0.23 GB read +
-# written.  The full workload is ten such ranges and every kind's traffic grows in proportion to
+# workload that fills one range of whole sequences (--prompts 1 --samples 26 --seed 2: 64,704 live
+# tokens, same d and V): logits 19.69 + 20.06 GB, dW 49.90 + 2.18 GB, dH 47.43 + 0.45 GB read +
+# written.  The full workload is five such ranges and every kind's traffic grows in proportion to
 # the ranges it processes, so a step's figure is this times its live tokens.
-DRAM_BYTES_PER_TOKEN_7B = 73.73e9 / 32634
+DRAM_BYTES_PER_TOKEN_7B = 139.70e9 / 64704
 
 
 # ---------------------------------------------------------------------------- helpers
@@ -432,7 +432,7 @@ def run_cuda(args) -> None:
                 # capture times this step's live tokens; only for the workload and path it was taken on
                 "traffic": (DRAM_BYTES_PER_TOKEN_7B * n_live
                             if (DRAM_BYTES_PER_TOKEN_7B and fused and not grpo and args.workload == "7b") else None),
-                "traffic_kind": "scaled by live tokens from a reduced capture (one range of 32,634 tokens, same d and V)",
+                "traffic_kind": "scaled by live tokens from a reduced capture (one range of 64,704 tokens, same d and V)",
                 "peak_kind": f"bf16_tflops_sustained of {peaks['source']}",
                 "credited_tflops": flops_step / (ms_step * 1e-3) / 1e12,
                 "credited_frac_of_sustained": flops_step / (ms_step * 1e-3) / 1e12 / peaks["sustained"],
