@@ -265,6 +265,22 @@ int oapl_adamw_step(void* W, float* master, const float* dW, float* m, float* v,
 int oapl_entropy(const oapl_problem* problem /*host*/, float* token_entropy, float* seq_entropy,
                  float* mean_entropy, void* ws, size_t ws_bytes, int flags, void* stream);
 
+/*
+ * Scalars a trainer logs next to the loss, from the quantities of Eq. 2 / Eq. 3 that the last
+ * loss forward (oapl_loss_fwd, oapl_loss_fwd_bwd, oapl_loss_fwd_bwd_ex) left in `ws`; nothing is
+ * recomputed.  With D_i = ln pi(y_i|x) - ln pi_vllm(y_i|x) and A_i = r_i - vhat[g_i]:
+ *   stats[0] response tokens of the batch         stats[4] mean A_i over all rollouts
+ *   stats[1] mean |D_i| over the rollouts with    stats[5] fraction of the groups (with members)
+ *            response tokens                               whose rewards are all equal (A_i = 0)
+ *   stats[2] max |D_i| over the same rollouts     stats[6] mean reward
+ *   stats[3] sum_i D_i / response tokens          stats[7] 0
+ * stats: 8 floats on the device; vhat [P]: the forward's output.  `problem`, `ws`, `ws_bytes`
+ * and `flags` are those of the forward (OAPL_FLAG_FUSED for the single calls).  Without a
+ * preceding loss forward on `ws` the status word becomes OAPL_ERR_BAD_STATE.
+ */
+int oapl_batch_stats(const oapl_problem* problem /*host*/, const float* vhat, float* stats, void* ws,
+                     size_t ws_bytes, int flags, void* stream);
+
 /* Synchronises `stream` and returns the status word the device recorded in `ws`
  * since the last forward call (OAPL_OK if none). */
 int oapl_get_last_status(void* ws, void* stream);

@@ -152,6 +152,40 @@ def loss_from_sums(D, reward, group_id, P, beta_v, beta_loss, loss_scale):
     return dict(loss=loss, vhat=vhat, A=A, delta=delta, coef=coef)
 
 
+def batch_stats(D, T, reward, group_id, vhat, P):
+    """Diagnostics of one batch from the quantities of Eq. 2 / Eq. 3 (the paper tracks training
+    curves; these are the scalars a trainer would log next to the loss):
+
+      live_tokens            sum_i T_i
+      mean_abs_log_ratio     mean over the sequences with T_i > 0 of |D_i|,  D_i = ln pi/pi_vllm (y_i|x)
+      max_abs_log_ratio      max over the same sequences of |D_i|
+      mean_token_log_ratio   sum_i D_i / sum_i T_i
+      mean_advantage         mean over all sequences of A_i = r_i - V^_{g(i)}  (text below Eq. 2)
+      frac_groups_all_equal  fraction of the groups with members whose rewards are all equal
+                             (there A_i = 0: the term of Eq. 3 only pulls the log-ratio to 0)
+      mean_reward            mean over all sequences of r_i
+    Empty denominators give 0.
+    """
+    D = np.asarray(D, dtype=np.float64)
+    T = np.asarray(T, dtype=np.float64)
+    r = np.asarray(reward, dtype=np.float64)
+    g = np.asarray(group_id).astype(np.int64)
+    vhat = np.asarray(vhat, dtype=np.float64)
+    live = T > 0
+    n_live = T.sum()
+    groups = [r[g == p] for p in range(P)]
+    with_members = [x for x in groups if x.size]
+    return dict(
+        live_tokens=float(n_live),
+        mean_abs_log_ratio=float(np.abs(D[live]).mean()) if live.any() else 0.0,
+        max_abs_log_ratio=float(np.abs(D[live]).max()) if live.any() else 0.0,
+        mean_token_log_ratio=float(D[live].sum() / n_live) if n_live > 0 else 0.0,
+        mean_advantage=float((r - vhat[g]).mean()) if r.size else 0.0,
+        frac_groups_all_equal=(sum(1 for x in with_members if x.max() == x.min()) / len(with_members)
+                               if with_members else 0.0),
+        mean_reward=float(r.mean()) if r.size else 0.0)
+
+
 def loss_fwd(H, W, targets, mask, seq_id, group_id, reward, logp_inf,
              S, P, beta_v, beta_loss, loss_scale):
     """Whole forward: token log-probs -> sequence sums -> Eq. 2 -> Eq. 3."""

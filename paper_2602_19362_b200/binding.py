@@ -25,7 +25,7 @@ EXPORTS = ["oapl_workspace_bytes", "oapl_token_logprobs", "oapl_value_estimate",
            "oapl_status_string", "oapl_debug_gemm", "oapl_profile_enable", "oapl_profile_read",
            "oapl_token_logprobs_static", "oapl_loss_fwd_bwd", "oapl_profile_read_clocks", "oapl_entropy", "oapl_group_advantage",
            "oapl_grpo_loss_fwd_bwd", "oapl_adamw_workspace_bytes", "oapl_adamw_step", "oapl_loss_fwd_bwd_ex",
-           "oapl_get_range_count", "oapl_profile_applies", "oapl_range_slots"]
+           "oapl_get_range_count", "oapl_profile_applies", "oapl_range_slots", "oapl_batch_stats"]
 
 
 class OaplProblem(ctypes.Structure):
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(OaplCallOptions), vp]
         L.oapl_get_range_count.restype = i32
         L.oapl_get_range_count.argtypes = [vp, vp]
+        L.oapl_batch_stats.restype = i32
+        L.oapl_batch_stats.argtypes = [pp, vp, vp, vp, sz, i32, vp]
         L.oapl_range_slots.restype = i32
         L.oapl_range_slots.argtypes = [i64, i64, ctypes.c_int32, ctypes.c_int32]
         L.oapl_profile_applies.restype = i32
@@ -226,6 +228,17 @@ def oapl_entropy(problem, token_entropy, seq_entropy, mean_entropy, ws, flags=0)
                             _ptr(ws), ws.numel(), flags, _stream())
     if rc != OAPL_OK:
         raise OaplError(rc, "oapl_entropy")
+
+
+STATS = ("live_tokens", "mean_abs_log_ratio", "max_abs_log_ratio", "mean_token_log_ratio", "mean_advantage",
+         "frac_groups_all_equal", "mean_reward")
+
+
+def oapl_batch_stats(problem, vhat, stats, ws, flags=0):
+    rc = lib().oapl_batch_stats(ctypes.byref(problem), _ptr(vhat), _ptr(stats), _ptr(ws), ws.numel(), flags,
+                                _stream())
+    if rc != OAPL_OK:
+        raise OaplError(rc, "oapl_batch_stats")
 
 
 def oapl_get_last_status(ws) -> int:

@@ -188,6 +188,32 @@ struct Tile {
   int first, last, split;
 };
 
+// Tile number pid + j * npairs of an MB x NB grid of 256-row tiles, NACC * 256 columns wide, handed
+// out round-robin.  When the last, partial round holds r tiles and 2 r <= npairs, that round hands
+// them out as 2 r half-width tiles (one accumulator each), so it takes half as long.
+template <int NACC>
+__device__ __forceinline__ bool grid_tile(int MB, int NB, int ncols, int pid, int npairs, int j, int& mb,
+                                          int& n0, int& nh) {
+  constexpr int kTN = NACC * kBN;
+  const int total = MB * NB;
+  const int full = (total / npairs) * npairs, r = total - full;
+  const int tix = pid + j * npairs;
+  if (NACC == 2 && tix >= full && r > 0 && 2 * r <= npairs) {
+    const int q = tix - full;
+    if (q >= 2 * r) return false;
+    const int tt = full + (q >> 1);
+    mb = tt / NB;
+    n0 = (tt % NB) * kTN + (q & 1) * kBN;
+    nh = 1;
+    return n0 < ncols;
+  }
+  if (tix >= total) return false;
+  mb = tix / NB;
+  n0 = (tix % NB) * kTN;
+  nh = (NACC == 2 && n0 + kBN < ncols) ? 2 : 1;
+  return true;
+}
+
 // Tile j of this CTA pair for rows [row_begin, row_end) of the compacted row space.
 // m0 is the pair's first row; CTA `rank` of the pair owns rows m0 + 128*rank ....
 template <int MODE, int NACC>
@@ -239,33 +265,27 @@ __device__ __forceinline__ bool get_tile(const GemmParams& p, int row_begin, int
   } else if (MODE == MODE_DH) {
     if (rows <= 0) return false;
     const int MB = (rows + kTileM - 1) / kTileM, NB = (p.d + kTN - 1) / kTN;
-    const int tix = pid + j * npairs;
-    if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kTileM;  // row inside the staged chunk
-    t.n0 = (tix % NB) * kTN;
-    t.nh = (NACC == 2 && t.n0 + kBN < p.d) ? 2 : 1;
+    int mb;
+    if (!grid_tile<NACC>(MB, NB, p.d, pid, npairs, j, mb, t.n0, t.nh)) return false;
+    t.m0 = mb * kTileM;  // row inside the staged chunk
     t.ka0 = t.kb0 = 0;
     t.nk = (p.V + kBK - 1) / kBK;
     return true;
   } else if (MODE == MODE_DW) {
     if (rows <= 0) return false;
     const int MB = (p.V + kTileM - 1) / kTileM, NB = (p.d + kTN - 1) / kTN;
-    const int tix = pid + j * npairs;
-    if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kTileM;  // vocabulary row
-    t.n0 = (tix % NB) * kTN;
-    t.nh = (NACC == 2 && t.n0 + kBN < p.d) ? 2 : 1;
-    t.ka0 = 0;          // staged chunk rows are range-relative
-    t.kb0 = row_begin;  // compacted H rows are absolute
+    int mb;
+    if (!grid_tile<NACC>(MB, NB, p.d, pid, npairs, j, mb, t.n0, t.nh)) return false;
+    t.m0 = mb * kTileM;  // vocabulary row
+    t.ka0 = 0;           // staged chunk rows are range-relative
+    t.kb0 = row_begin;   // compacted H rows are absolute
     t.nk = (rows + kBK - 1) / kBK;
     return true;
   } else {
     const int MB = (p.M + kTileM - 1) / kTileM, NB = (p.N + kTN - 1) / kTN;
-    const int tix = pid + j * npairs;
-    if (tix >= MB * NB) return false;
-    t.m0 = (tix / NB) * kTileM;
-    t.n0 = (tix % NB) * kTN;
-    t.nh = (NACC == 2 && t.n0 + kBN < p.N) ? 2 : 1;
+    int mb;
+    if (!grid_tile<NACC>(MB, NB, p.N, pid, npairs, j, mb, t.n0, t.nh)) return false;
+    t.m0 = mb * kTileM;
     t.ka0 = t.kb0 = 0;
     t.nk = p.K / kBK;
     return true;

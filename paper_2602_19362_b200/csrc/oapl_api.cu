@@ -899,6 +899,25 @@ int oapl_entropy(const oapl_problem* p, float* token_entropy, float* seq_entropy
   return OAPL_OK;
 }
 
+int oapl_batch_stats(const oapl_problem* p, const float* vhat, float* stats, void* ws, size_t ws_bytes, int flags,
+                     void* stream) {
+  int rc = check_problem(p, true);
+  if (rc != OAPL_OK) return rc;
+  if (!vhat || !stats || !ws) return OAPL_ERR_INVALID_ARG;
+  if ((uintptr_t)ws & 1023) return OAPL_ERR_MISALIGNED;
+  Carve c;
+  if (!carve(p, flags, &c)) return OAPL_ERR_INVALID_ARG;
+  if (ws_bytes < c.total) return OAPL_ERR_WORKSPACE_TOO_SMALL;
+  uint8_t* w = static_cast<uint8_t*>(ws);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  batch_stats_kernel<<<1, 256, 0, st>>>(reinterpret_cast<const float*>(w + c.seq_D),
+                                        reinterpret_cast<const int*>(w + c.cstart),
+                                        reinterpret_cast<const int*>(w + c.cend), p->reward, p->group_id, vhat,
+                                        p->S, p->P, reinterpret_cast<DevState*>(w + c.state), stats);
+  CKL();
+  return OAPL_OK;
+}
+
 int oapl_profile_enable(int on) {
   if (!on) {
     g_prof.device = -1;

@@ -604,6 +604,90 @@ __global__ void grpo_loss_kernel(const float* __restrict__ seq_obj, const int* _
 }
 
 // =====================================================================================
+// Batch diagnostics from what a loss forward left in the workspace (one CTA, fixed order).
+// =====================================================================================
+// stats[0] live tokens, [1] mean |D_i| and [2] max |D_i| over the sequences with response tokens,
+// [3] sum D_i / live tokens, [4] mean advantage r_i - vhat[g_i], [5] fraction of the groups with
+// members whose rewards are all equal, [6] mean reward, [7] 0.
+constexpr int kStatsCount = 8;
+__global__ void batch_stats_kernel(const float* __restrict__ seq_D, const int* __restrict__ cstart,
+                                   const int* __restrict__ cend, const float* __restrict__ reward,
+                                   const int* __restrict__ group_id, const float* __restrict__ vhat, int S, int P,
+                                   DevState* st, float* __restrict__ stats) {
+  __shared__ double sh[4][8];
+  __shared__ float shmax[8];
+  __shared__ int shcnt[3][8];
+  if (st->fwd_tag != 0x0A91) {
+    if (threadIdx.x == 0) set_error(&st->status, -10);
+    return;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  double sum_abs = 0.0, sum_d = 0.0, sum_adv = 0.0, sum_r = 0.0;
+  float max_abs = 0.f;
+  int n_seq_live = 0;
+  for (int i = threadIdx.x; i < S; i += blockDim.x) {
+    const float r = reward[i];
+    const int g = group_id[i];
+    sum_r += (double)r;
+    sum_adv += (double)r - (double)((g >= 0 && g < P) ? vhat[g] : 0.f);
+    if (cend[i] > cstart[i]) {
+      const float dd = seq_D[i];
+      sum_abs += fabs((double)dd);
+      sum_d += (double)dd;
+      max_abs = fmaxf(max_abs, fabsf(dd));
+      ++n_seq_live;
+    }
+  }
+  // groups: one warp per group in turn; all-equal when the members' minimum equals their maximum
+  int n_groups = 0, n_equal = 0;
+  for (int p = warp; p < P; p += nwarps) {
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = lane; i < S; i += 32)
+      if (group_id[i] == p) { lo = fminf(lo, reward[i]); hi = fmaxf(hi, reward[i]); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (hi >= lo) { ++n_groups; n_equal += (hi == lo) ? 1 : 0; }   // same value in every lane
+  }
+  sum_abs = warp_sum_d(sum_abs);
+  sum_d = warp_sum_d(sum_d);
+  sum_adv = warp_sum_d(sum_adv);
+  sum_r = warp_sum_d(sum_r);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    max_abs = fmaxf(max_abs, __shfl_down_sync(0xffffffffu, max_abs, o));
+    n_seq_live += __shfl_down_sync(0xffffffffu, n_seq_live, o);
+  }
+  if (lane == 0) {
+    sh[0][warp] = sum_abs; sh[1][warp] = sum_d; sh[2][warp] = sum_adv; sh[3][warp] = sum_r;
+    shmax[warp] = max_abs;
+    shcnt[0][warp] = n_seq_live; shcnt[1][warp] = n_groups; shcnt[2][warp] = n_equal;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t[4] = {0.0, 0.0, 0.0, 0.0};
+    float mx = 0.f;
+    int c[3] = {0, 0, 0};
+    for (int w = 0; w < nwarps; ++w) {
+      for (int k = 0; k < 4; ++k) t[k] += sh[k][w];
+      mx = fmaxf(mx, shmax[w]);
+      for (int k = 0; k < 3; ++k) c[k] += shcnt[k][w];
+    }
+    const int n_live = st->n_live;
+    stats[0] = (float)n_live;
+    stats[1] = c[0] > 0 ? (float)(t[0] / (double)c[0]) : 0.f;
+    stats[2] = mx;
+    stats[3] = n_live > 0 ? (float)(t[1] / (double)n_live) : 0.f;
+    stats[4] = S > 0 ? (float)(t[2] / (double)S) : 0.f;
+    stats[5] = c[1] > 0 ? (float)((double)c[2] / (double)c[1]) : 0.f;
+    stats[6] = S > 0 ? (float)(t[3] / (double)S) : 0.f;
+    stats[7] = 0.f;
+  }
+}
+
+// =====================================================================================
 // Policy-entropy statistic read back from what a forward left in the workspace.
 // =====================================================================================
 // One CTA per sequence: mean of the per-row entropies over the sequence's response tokens

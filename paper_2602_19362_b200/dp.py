@@ -66,8 +66,9 @@ def start_allreduce_dW(dW: torch.Tensor, dW_ready=None, comm_stream=None, group=
     `dW_ready` (a torch.cuda.Event) at that point.  On CUDA tensors the all-reduce is enqueued
     on `comm_stream` behind that event, so NCCL runs under the remaining compute; on CPU
     tensors (gloo) it is started asynchronously at once.  Returns a handle for
-    finish_allreduce; None without a process group."""
-    if not dist.is_available() or not dist.is_initialized() or dist.get_world_size(group) == 1:
+    finish_allreduce; None without a process group.  (A group of one rank still goes through the
+    same streams and events; the sum is then the identity.)"""
+    if not dist.is_available() or not dist.is_initialized():
         return None
     if dW.is_cuda:
         if dW_ready is None or comm_stream is None:

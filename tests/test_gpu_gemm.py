@@ -11,8 +11,9 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("wide", [False, True], ids=["256x256", "256x512"])
 @pytest.mark.parametrize("a_mn,b_mn", [(0, 0), (0, 1), (1, 1), (1, 0)])
+# the last shape has 81 wide tiles for 74 CTA pairs: its partial second round is split into half-width tiles
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (384, 512, 320), (200, 264, 128), (1000, 1304, 1088),
-                                   (520, 3000, 4096)])
+                                   (520, 3000, 4096), (2304, 4608, 128)])
 def test_debug_gemm(M, N, K, a_mn, b_mn, wide):
     g = torch.Generator().manual_seed(M * 7 + N * 3 + K + a_mn * 2 + b_mn)
     A = torch.randn(M, K, generator=g).to(torch.bfloat16)

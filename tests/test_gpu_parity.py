@@ -80,3 +80,36 @@ def test_single_call_reports_a_sequence_longer_than_the_staging_capacity(monkeyp
     cpu = synth.make_batch(wl, seed=13)
     out = hp.run_gpu(hp.to_dev(cpu), fused=True)
     assert out["status"] == -11
+
+
+@BOTH
+def test_batch_stats_entry_point(fused):
+    from oracle import oapl_oracle as orc
+    cpu = synth.make_batch(synth.WORKLOADS["tiny"], seed=14)
+    cpu["mask"][cpu["seq_id"] == 3] = 0                  # a rollout without response tokens
+    cpu["reward"][4:8] = 1.0                             # a group with all-equal rewards
+    cpu["live_tokens"] = int(cpu["mask"].sum())
+    out = hp.run_gpu(hp.to_dev(cpu), fused=fused)
+    ref = hp.run_oracle(cpu)
+    hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
+    stats = torch.full((8,), float("nan"), device="cuda")
+    B.oapl_batch_stats(out["prob"], out["vhat"], stats, out["ws"], B.OAPL_FLAG_FUSED if fused else 0)
+    assert B.oapl_get_last_status(out["ws"]) == 0
+    want = orc.batch_stats(ref["D"], ref["T"], hp.npy(cpu["reward"]), hp.npy(cpu["group_id"]), ref["vhat"], cpu["P"])
+    got = dict(zip(B.STATS, hp.npy(stats)[:7].tolist()))
+    assert got["live_tokens"] == want["live_tokens"] and got["frac_groups_all_equal"] == want["frac_groups_all_equal"]
+    assert got["mean_reward"] == pytest.approx(want["mean_reward"], rel=1e-6)
+    assert got["mean_advantage"] == pytest.approx(want["mean_advantage"], rel=1e-5, abs=1e-6)
+    # the log-ratios inherit the error of the token log-probs: 5e-4 sqrt(T) per sequence (see helpers)
+    tol = 5e-4 * np.sqrt(ref["T"].max() + 1)
+    assert abs(got["mean_abs_log_ratio"] - want["mean_abs_log_ratio"]) <= tol
+    assert abs(got["max_abs_log_ratio"] - want["max_abs_log_ratio"]) <= tol
+    assert abs(got["mean_token_log_ratio"] - want["mean_token_log_ratio"]) <= hp.TOL_TOKEN
+    assert float(stats[7]) == 0.0
+    # without a loss forward on the workspace the call reports it
+    prob = out["prob"]
+    ws = B.alloc_workspace(prob, B.OAPL_FLAG_FUSED if fused else 0)
+    tok = torch.zeros(cpu["N"], device="cuda")
+    B.oapl_token_logprobs(prob, tok, None, ws)
+    B.oapl_batch_stats(prob, out["vhat"], stats, ws, B.OAPL_FLAG_FUSED if fused else 0)
+    assert B.oapl_get_last_status(ws) == -10

@@ -81,7 +81,9 @@ def test_no_entry_point_writes_outside_its_workspace_or_outputs():
     dH, dW = out((N, d), bf16), out((V, d), f32)
     B.oapl_loss_fwd(prob, loss, seq, vhat, delta, tok, ws)
     B.oapl_loss_bwd(prob, dH, dW, False, ws)
-    check(ws, "loss_fwd + loss_bwd")
+    stats = out((8,), f32)
+    B.oapl_batch_stats(prob, vhat, stats, ws)
+    check(ws, "loss_fwd + loss_bwd + batch_stats")
     want_dW = dW.clone()
     # single call, plain and with options, and the GRPO objective on the same pipeline
     wsf = workspace(B.OAPL_FLAG_FUSED)
@@ -231,3 +233,46 @@ def test_call_options_bounds_event_and_range_count(monkeypatch):
                            False, ws, B.make_options(0, 0, None))
     assert B.oapl_get_last_status(ws) == 0
     assert torch.equal(o["dW"], plain["dW"])
+
+
+def test_overlapped_exchange_plumbing_on_a_one_rank_nccl_group():
+    # The data-parallel step: oapl_loss_fwd_bwd_ex records the dW-ready event, a second stream waits
+    # for it and runs the NCCL all-reduce of dW while the compute stream finishes dH, then the loss
+    # follows.  With one rank the sums are identities, so dW and the loss must come out bit for bit
+    # as without the exchange; what is exercised is the event handle, the stream order and NCCL.
+    import os
+    import socket
+    import torch.distributed as dist
+    from paper_2602_19362_b200 import dp
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        wl = dataclasses.replace(synth.WORKLOADS["tiny"], prompts=16, samples=8, length=("uniform", 64, 256),
+                                 padded_to=256, d=256, V=4096 + 72)
+        cpu = synth.make_batch(wl, seed=15)
+        dev = hp.to_dev(cpu)
+        plain = hp.run_gpu(dev, fused=True)
+        prob, ws = plain["prob"], plain["ws"]
+        N, S, P, d, V = (cpu[k] for k in ("N", "S", "P", "d", "V"))
+        loss, seq = torch.zeros(1, device="cuda"), torch.zeros(S, device="cuda")
+        vhat, delta = torch.zeros(P, device="cuda"), torch.zeros(S, device="cuda")
+        dH = torch.empty(N, d, dtype=torch.bfloat16, device="cuda")
+        dW = torch.empty(V, d, device="cuda")
+        ev = torch.cuda.Event()
+        ev.record()
+        comm = torch.cuda.Stream()
+        opts = B.make_options(cpu["live_tokens"], int(cpu["lengths"].max()), ev)
+        for _ in range(3):                          # steps back to back, as in the timed loop
+            B.oapl_loss_fwd_bwd_ex(prob, loss, seq, vhat, delta, None, dH, dW, False, ws, opts)
+            handle = dp.start_allreduce_dW(dW, ev, comm)
+            assert handle is not None
+            dp.finish_allreduce(handle, loss)
+        torch.cuda.synchronize()
+        assert B.oapl_get_last_status(ws) == 0
+        assert torch.equal(dW, plain["dW"]) and torch.equal(loss, plain["loss"])
+        assert torch.equal(dH.view(torch.int16), plain["dH"].view(torch.int16))
+    finally:
+        dist.destroy_process_group()

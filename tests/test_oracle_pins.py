@@ -543,3 +543,43 @@ def test_gradients_match_torch_autograd():
     assert go["loss"] == pytest.approx(float(gloss.detach()), rel=1e-12)
     assert go["clipped"].any()
     assert np.allclose(dH, gH.numpy(), rtol=1e-9, atol=1e-12) and np.allclose(dW, gW.numpy(), rtol=1e-9, atol=1e-12)
+
+
+# --------------------------------------------------------------------------
+# batch diagnostics
+# --------------------------------------------------------------------------
+def test_batch_stats_on_a_hand_computed_example():
+    # four rollouts in two groups; the third has no response token and must not count in the
+    # log-ratio statistics; group 1 has all-equal rewards
+    D = [1.0, -3.0, 123.0, 2.0]
+    T = [2, 1, 0, 4]
+    st = orc.batch_stats(D, T, reward=[1.0, 0.0, 1.0, 1.0], group_id=[0, 0, 1, 1], vhat=[0.7, 1.0], P=3)
+    assert st["live_tokens"] == 7.0
+    assert st["mean_abs_log_ratio"] == pytest.approx(2.0, rel=1e-15)       # (1 + 3 + 2) / 3
+    assert st["max_abs_log_ratio"] == 3.0
+    assert st["mean_token_log_ratio"] == pytest.approx(0.0, abs=1e-15)     # (1 - 3 + 2) / 7
+    assert st["mean_advantage"] == pytest.approx(-0.1, rel=1e-12)          # (0.3 - 0.7 + 0 + 0) / 4
+    assert st["frac_groups_all_equal"] == 0.5                              # the empty third group is not counted
+    assert st["mean_reward"] == 0.75
+
+
+def test_batch_stats_mean_advantage_is_never_positive_with_the_value_estimate_of_eq2():
+    # V^ is a log-mean-exp, so V^_p >= mean of the group's rewards (Jensen): the advantages of a
+    # group sum to at most 0, with equality exactly when its rewards are all equal
+    rng = np.random.default_rng(3)
+    for beta in (0.1, 1.0, 10.0):
+        r = rng.normal(size=40)
+        g = rng.integers(0, 6, size=40)
+        vhat = orc.value_estimate(r, g, 7, beta)
+        st = orc.batch_stats(np.zeros(40), np.ones(40), r, g, vhat, 7)
+        assert st["mean_advantage"] < 0.0
+        assert st["frac_groups_all_equal"] <= 1.0 / 6 + 1e-12             # only a one-member group can be "equal"
+    r = np.repeat(rng.normal(size=5), 4)                                   # every group constant
+    g = np.repeat(np.arange(5), 4)
+    st = orc.batch_stats(np.zeros(20), np.ones(20), r, g, orc.value_estimate(r, g, 5, 0.5), 5)
+    assert st["mean_advantage"] == pytest.approx(0.0, abs=1e-12) and st["frac_groups_all_equal"] == 1.0
+
+
+def test_batch_stats_of_an_empty_batch_are_zero():
+    st = orc.batch_stats(np.zeros(3), np.zeros(3), np.zeros(3), np.zeros(3, dtype=int), np.zeros(1), 1)
+    assert st["live_tokens"] == 0 and st["mean_abs_log_ratio"] == 0 and st["mean_token_log_ratio"] == 0
