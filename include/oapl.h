@@ -57,6 +57,7 @@ typedef enum {
  *   OAPL_SPLITS        vocabulary splits per wave of the logits sweeps (chosen from the L2 budget)
  *   OAPL_L2_BUDGET_MB  L2 budget for the hidden-state blocks of one wave of a sweep (48)
  *   OAPL_ACC_SKEW      K-steps by which the second accumulator of a sweep tile trails the first (4)
+ *   OAPL_NVTX          1 = NVTX ranges around the phases a call enqueues, for a timeline profiler (0)
  *   OAPL_SYNC_EVERY    K-steps between the lock-step meetings of the CTA pairs (32; 0 = never)
  * They change workspace sizes and schedules, never results beyond summation order across splits.
  */

@@ -28,6 +28,9 @@
 //             half-accumulator order hides: the epilogue drains accumulator 0 first and
 //             releases it, and the UMMA thread starts the next tile with accumulator 0's
 //             share of the first four K-steps while accumulator 1 is still being drained.
+//             In the vocabulary sweeps the end of a tile is skewed the same way: the last four
+//             K-steps are issued for accumulator 0 first, which goes to the epilogue on its own
+//             barrier while accumulator 1's share of those K-steps still runs.
 //             dH (K = V) and dW (K = rows of the range) have long K loops and four epilogue
 //             warps; dW leaves through TMA reduce-add.  The vocabulary sweeps (short K = d,
 //             an exponential per element, bf16 stores in two of the three) have eight.

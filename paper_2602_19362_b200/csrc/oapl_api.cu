@@ -2,6 +2,7 @@
 // workspace carve-up, tensor-map encoding and the launch sequences.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <atomic>
 #include <cmath>
@@ -43,6 +44,20 @@ static int env_int(const char* name, int dflt) {
   const char* s = getenv(name);
   return (s && *s) ? atoi(s) : dflt;
 }
+
+// Named ranges for a timeline profiler around the phases a call enqueues (OAPL_NVTX=1; off by
+// default).  They mark host-side enqueue spans; the profiler attributes the launches inside.
+struct NvtxRange {
+  bool on;
+  explicit NvtxRange(const char* name) : on(env_int("OAPL_NVTX", 0) != 0) {
+    if (on) nvtxRangePushA(name);
+  }
+  ~NvtxRange() {
+    if (on) nvtxRangePop();
+  }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 static bool carve(const oapl_problem* p, int flags, Carve* c) {
   if (!p || p->N <= 0 || p->d <= 0 || p->V <= 0 || p->S <= 0 || p->P <= 0) return false;
@@ -339,6 +354,7 @@ static int check_problem(const oapl_problem* p, bool need_loss_inputs) {
 // compacted-sequence bounds and the dense copy of the live rows of H.
 static int prologue(const oapl_problem* p, const Carve& c, uint8_t* ws, float* token_logp, bool with_q,
                     cudaStream_t st) {
+  NvtxRange nvtx("oapl: live-row compaction");
   const int n_sm = sm_count();
   if (n_sm <= 0) return OAPL_ERR_CUDA;
   DevState* state = reinterpret_cast<DevState*>(ws + c.state);
@@ -411,6 +427,7 @@ static int forward_common(const oapl_problem* p, const Carve& c, uint8_t* ws, fl
   gp.tgt_c = tgt_c;
   gp.err = &state->status;
   set_lockstep(&gp, ws, c, 0, p->d / kBK);
+  NvtxRange nvtx("oapl: logits + online log-sum-exp, merge, sequence sums");
   int rc = launch_gemm<MODE_LSE, 0, 0, 2>(tmA, tmB, tmA, gp, 2 * gp.R * gp.C, st);
   if (rc != OAPL_OK) return rc;
 
@@ -548,6 +565,7 @@ static int staged_fwd_bwd(const oapl_problem* p, const Objective& ob, float* los
   // slots come first (their launches return at once) and the last slot always holds the last
   // range: the event after its dW launch marks dW complete while its dH contraction still runs.
   for (int k = 0; k < slots; ++k) {
+    NvtxRange nvtx("oapl: range slot (logits + exp, coefficients, dW, dH)");
     const RangeRec* rg = ranges + k;
     gp.range_ptr = &rg->row_begin;
     gp.rowscale = nullptr;
@@ -758,6 +776,7 @@ int oapl_loss_bwd(const oapl_problem* p, void* dH, float* dW, int accumulate_dW,
   CK(cudaMemsetAsync(w + c.sync, 0, 4 * (size_t)kSyncSlots, st));
   int slot = 0;
   for (int r0 = 0; r0 < c.n_pad; r0 += c.chunk_rows) {
+    NvtxRange nvtx("oapl: backward row chunk (logit gradient, dH, dW)");
     gp.row_begin = r0;
     set_lockstep(&gp, w, c, slot++, p->d / kBK);
     rc = launch_gemm<MODE_GRAD, 0, 0, 2>(tmH, tmW, tmGst, gp, 2 * gp.R * gp.C, st);

@@ -53,6 +53,7 @@ def run_gpu(dev, beta_v=None, beta_loss=None, loss_scale=None, backward=True, ac
     out["n_live"] = B.oapl_get_live_rows(ws)
     out["ws"] = ws
     out["prob"] = prob
+    out["batch"] = dev          # the problem struct points into these tensors: keep them alive with it
     return out
 
 

@@ -168,3 +168,14 @@ def test_two_streams_with_their_own_workspaces_give_the_single_stream_results():
         for k in ("loss", "seq_logp", "token_logp", "dW"):
             assert torch.equal(o[k], w[k]), k
         assert torch.equal(o["dH"].view(torch.int16), w["dH"].view(torch.int16))
+
+
+def test_nvtx_ranges_do_not_change_anything(monkeypatch):
+    dev = hp.to_dev(synth.make_batch(TINY, seed=3))
+    want = [hp.run_gpu(dev, fused=f) for f in (False, True)]
+    monkeypatch.setenv("OAPL_NVTX", "1")
+    for f, w in zip((False, True), want):
+        got = hp.run_gpu(dev, fused=f)
+        assert got["status"] == 0
+        for k in ("loss", "seq_logp", "token_logp", "dW"):
+            assert torch.equal(got[k], w[k]), k

@@ -89,7 +89,8 @@ def test_batch_stats_entry_point(fused):
     cpu["mask"][cpu["seq_id"] == 3] = 0                  # a rollout without response tokens
     cpu["reward"][4:8] = 1.0                             # a group with all-equal rewards
     cpu["live_tokens"] = int(cpu["mask"].sum())
-    out = hp.run_gpu(hp.to_dev(cpu), fused=fused)
+    dev = hp.to_dev(cpu)                                 # the problem struct points into these tensors
+    out = hp.run_gpu(dev, fused=fused)
     ref = hp.run_oracle(cpu)
     hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
     stats = torch.full((8,), float("nan"), device="cuda")
