@@ -23,7 +23,6 @@ import os
 import statistics
 import subprocess
 import sys
-import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -35,10 +34,10 @@ UNIT = "tokens/s"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per live token of the single call's
 # three contraction kinds: one ncu capture of one launch per kind on a reduced copy of the 7B
 # workload that fills one range of whole sequences (--prompts 1 --samples 26 --seed 2: 64,704 live
-# tokens, same d and V): logits 19.69 + 20.06 GB, dW 49.90 + 2.18 GB, dH 47.43 + 0.45 GB read +
+# tokens, same d and V): logits 19.99 + 20.06 GB, dW 49.90 + 2.17 GB, dH 47.43 + 0.45 GB read +
 # written.  The full workload is five such ranges and every kind's traffic grows in proportion to
 # the ranges it processes, so a step's figure is this times its live tokens.
-DRAM_BYTES_PER_TOKEN_7B = 139.70e9 / 64704
+DRAM_BYTES_PER_TOKEN_7B = 140.00e9 / 64704
 
 
 # ---------------------------------------------------------------------------- helpers
@@ -78,7 +77,6 @@ def reduce_sum(value: float, dist, device) -> float:
 def oracle_sample(workload: str, live_rows: int):
     """A bounded sample of the workload for the CPU oracle: same d, V, distributions and
     betas, 2 prompts x 4 rollouts and about `live_rows` response tokens."""
-    import numpy as np
     from oracle import oapl_oracle as orc
     from paper_2602_19362_b200 import synth
     wl = synth.small_variant(workload, prompts=2, samples=4, live_rows=live_rows) \

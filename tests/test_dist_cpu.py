@@ -46,7 +46,6 @@ def test_identity_without_process_group():
 def _dp_worker(rank, world, port, q):
     sys.path.insert(0, ROOT)
     import numpy as np
-    from oracle import oapl_oracle as orc
     from paper_2602_19362_b200 import dp, synth
     from tests import helpers_cpu as hc
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))

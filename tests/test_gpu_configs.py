@@ -3,7 +3,6 @@ distributions, reward structure, noise level and temperatures as the full
 configuration, but 2 prompts x 4 rollouts and a few hundred response tokens, which the
 fp64 oracle finishes in seconds.  The rows still span several 128-row tiles with a
 ragged tail and the vocabulary spans ~600 tiles with (for V = 151936) a half tile."""
-import numpy as np
 import pytest
 
 from oracle import oapl_oracle as orc
