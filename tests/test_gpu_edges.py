@@ -179,3 +179,31 @@ def test_nvtx_ranges_do_not_change_anything(monkeypatch):
         assert got["status"] == 0
         for k in ("loss", "seq_logp", "token_logp", "dW"):
             assert torch.equal(got[k], w[k]), k
+
+
+@pytest.mark.parametrize("d,V", [(64, 7), (128, 255), (64, 256), (192, 257), (64, 511), (128, 512), (64, 513),
+                                 (320, 1025), (64, 2049)])
+def test_vocabulary_sizes_around_the_tile_boundaries(d, V):
+    # 256 and 512 are the widths of one accumulator and of one sweep tile: sizes just below, at and
+    # just above them, on both paths, with a handful of short sequences (one partial row block)
+    wl = dataclasses.replace(TINY, prompts=2, samples=3, length=("uniform", 3, 40), padded_to=48, d=d, V=V)
+    cpu = synth.make_batch(wl, seed=d + V)
+    ref = hp.run_oracle(cpu)
+    for fused in (False, True):
+        hp.assert_parity(hp.run_gpu(hp.to_dev(cpu), fused=fused), ref, hp.npy(cpu["mask"]))
+
+
+@pytest.mark.parametrize("rows", [1, 127, 128, 129, 257])
+def test_row_counts_around_the_row_block(rows):
+    # two rollouts of one prompt with `rows` response tokens each: the live rows end just below, at
+    # and just above a 256-row block (2, 254, 256, 258, 514); unequal rewards keep the residual of
+    # Eq. 3 away from a pure cancellation, so the loss tolerance means something
+    wl = dataclasses.replace(TINY, prompts=1, samples=2, length=("uniform", rows, rows), padded_to=rows, d=128,
+                             V=700)
+    cpu = synth.make_batch(wl, seed=rows)
+    cpu["reward"][:] = torch.tensor([1.0, 0.0])
+    ref = hp.run_oracle(cpu)
+    for fused in (False, True):
+        out = hp.run_gpu(hp.to_dev(cpu), fused=fused)
+        assert out["n_live"] == 2 * rows
+        hp.assert_parity(out, ref, hp.npy(cpu["mask"]))
