@@ -276,3 +276,36 @@ def test_overlapped_exchange_plumbing_on_a_one_rank_nccl_group():
         assert torch.equal(dH.view(torch.int16), plain["dH"].view(torch.int16))
     finally:
         dist.destroy_process_group()
+
+
+def test_two_prompt_shards_run_one_after_the_other_sum_to_the_unsharded_step():
+    # The data-parallel step on the CUDA path without a second GPU: the two ranks' shards (whole
+    # groups, global loss_scale) are run one after the other on this GPU as independent calls, and
+    # their dW and loss are added as the all-reduce would.  Against the unsharded call only the
+    # summation order differs; against the oracle the stated tolerances hold.
+    from paper_2602_19362_b200 import dp
+    wl = dataclasses.replace(synth.WORKLOADS["tiny"], prompts=6, samples=4, length=("uniform", 20, 120),
+                             padded_to=128, d=256, V=4096 + 72)
+    cpu = synth.make_batch(wl, seed=17)
+    ref = hp.run_oracle(cpu)
+    whole = hp.run_gpu(hp.to_dev(cpu), fused=True)
+    hp.assert_parity(whole, ref, hp.npy(cpu["mask"]))
+    dW = torch.zeros_like(whole["dW"])
+    loss = 0.0
+    dH_rows, n_rows = [], 0
+    for rank in range(2):
+        shard = dp.shard_by_prompt(cpu, rank, 2)
+        out = hp.run_gpu(hp.to_dev(shard), fused=True)
+        assert out["status"] == 0 and out["n_live"] == shard["live_tokens"]
+        dW += out["dW"]
+        loss += float(out["loss"])
+        dH_rows.append(out["dH"])
+        n_rows += shard["N"]
+    assert n_rows == cpu["N"]
+    assert loss == pytest.approx(float(whole["loss"]), rel=1e-5)
+    assert loss == pytest.approx(ref["loss"], rel=hp.TOL_REL)
+    assert hp.fro_rel(hp.npy(dW), hp.npy(whole["dW"])) <= 1e-4
+    assert hp.fro_rel(hp.npy(dW), ref["dW"]) <= hp.TOL_FRO
+    dH = torch.cat(dH_rows).float()
+    assert hp.fro_rel(hp.npy(dH), hp.npy(whole["dH"].float())) <= 2e-3      # bf16 outputs of slightly different sums
+    assert hp.fro_rel(hp.npy(dH), ref["dH"]) <= hp.TOL_FRO
