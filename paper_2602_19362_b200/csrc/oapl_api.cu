@@ -208,10 +208,11 @@ static int sm_count() {
 // H row blocks within an L2 budget; a short row range is handled by the tail-wave
 // re-splitting of the schedule itself.
 // The budget: every H block is re-read by its C pairs for each vocabulary tile and has to stay
-// in L2 for a whole sweep.  DRAM counters show that blocks read by pairs in both halves of the
-// chip take room in both halves of the 126 MB L2: with 68 MB of blocks (R = 37 at d = 3584) half
-// of the re-reads went to DRAM (22 GB read per 32 k rows against 4 GB needed), with 33 MB
-// (R = 18) almost none (10 GB against 8).
+// in L2 for a whole sweep.  DRAM counters of the sweep on 32 k rows at d = 3584: with 68 MB of
+// blocks, each read by two pairs (R = 37, C = 2), half of the re-reads went to DRAM (22 GB read
+// against 4 GB needed); the same 68 MB read by one pair per block stayed resident (5.9 GB); 33 MB
+// read by four pairs each (R = 18, C = 4) stayed resident too (10 GB against 8).  So blocks with
+// several readers get about half of the 126 MB L2.
 constexpr int kL2BudgetMB = 48;
 static void pick_sweep(int n_sm, int d, int vtiles, int* R, int* C) {
   const int pairs = n_sm / 2;
