@@ -583,3 +583,51 @@ def test_batch_stats_mean_advantage_is_never_positive_with_the_value_estimate_of
 def test_batch_stats_of_an_empty_batch_are_zero():
     st = orc.batch_stats(np.zeros(3), np.zeros(3), np.zeros(3), np.zeros(3, dtype=int), np.zeros(1), 1)
     assert st["live_tokens"] == 0 and st["mean_abs_log_ratio"] == 0 and st["mean_token_log_ratio"] == 0
+
+
+# --------------------------------------------------------------------------
+# symmetries of the softmax LM head (index mistakes break them)
+# --------------------------------------------------------------------------
+def _step(p, beta_v=0.9, beta_loss=0.6, lam=0.5):
+    out = _fwd(p, beta_v, beta_loss, lam)
+    dH, dW = orc.loss_bwd(p["H"], p["W"], p["targets"], p["mask"], p["seq_id"], out["coef"])
+    return out, dH, dW
+
+
+def test_adding_one_vector_to_every_row_of_W_changes_nothing():
+    # every logit of a row moves by the same h . u, so the next-token distribution, the loss and g are
+    # unchanged; rows of g sum to zero, so dH = g.(W + 1 u^T) = g.W, and dW = g^T.H does not see W
+    p = _problem(seed=21)
+    u = np.random.default_rng(5).normal(size=p["W"].shape[1])
+    q = dict(p, W=p["W"] + u[None, :])
+    (a, dHa, dWa), (b, dHb, dWb) = _step(p), _step(q)
+    assert np.allclose(a["token_logp"], b["token_logp"], atol=1e-12)
+    assert a["loss"] == pytest.approx(b["loss"], rel=1e-11)
+    assert np.allclose(dHa, dHb, atol=1e-11) and np.allclose(dWa, dWb, atol=1e-11)
+
+
+def test_permuting_the_vocabulary_permutes_dW_and_nothing_else():
+    p = _problem(seed=22)
+    V = p["W"].shape[0]
+    perm = np.random.default_rng(6).permutation(V)          # new row j holds old row perm[j]
+    inv = np.argsort(perm)
+    q = dict(p, W=p["W"][perm], targets=inv[p["targets"]])
+    (a, dHa, dWa), (b, dHb, dWb) = _step(p), _step(q)
+    assert np.allclose(a["token_logp"], b["token_logp"], atol=1e-12)
+    assert a["loss"] == pytest.approx(b["loss"], rel=1e-12)
+    assert np.allclose(dHa, dHb, atol=1e-12)
+    assert np.allclose(dWa[perm], dWb, atol=1e-12)
+
+
+def test_renumbering_the_groups_and_scaling_the_loss():
+    # Eq. 2 / Eq. 3 see a group only as a set of rollouts: renumbering the groups changes nothing;
+    # the loss and both gradients are linear in loss_scale
+    p = _problem(seed=23, S=8, P=3)
+    q = dict(p, group_id=(2 - p["group_id"]))
+    (a, dHa, dWa), (b, dHb, dWb) = _step(p), _step(q)
+    assert a["loss"] == pytest.approx(b["loss"], rel=1e-13)
+    assert np.allclose(a["vhat"], b["vhat"][::-1], atol=1e-13)
+    assert np.allclose(dHa, dHb, atol=1e-13) and np.allclose(dWa, dWb, atol=1e-13)
+    c, dHc, dWc = _step(p, lam=1.5)
+    assert c["loss"] == pytest.approx(3.0 * a["loss"], rel=1e-13)
+    assert np.allclose(dHc, 3.0 * dHa, atol=1e-13) and np.allclose(dWc, 3.0 * dWa, atol=1e-13)
